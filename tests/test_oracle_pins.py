@@ -482,7 +482,7 @@ def test_noise_streams_feed_the_documented_stages():
     x = O.sample_runtimes(w, np.full((W, n), 0.5), seed, step, k)
     sd_q = np.log1p(np.exp(w["bsig"].astype(np.float64)))
     want = (w["bmu"].astype(np.float64) + sd_q * O.normals(seed, step, W - 1, k, n)
-            + 0.5 * O.normals(seed, step, O.STREAM_TRANSITION, k, n)
-            + 0.25 * O.normals(seed, step, O.STREAM_EMISSION, k, n))
+            + math.exp(0.5 * float(w["b2"][n])) * O.normals(seed, step, O.STREAM_TRANSITION, k, n)
+            + math.exp(0.5 * float(w["b4"][n])) * O.normals(seed, step, O.STREAM_EMISSION, k, n))
     assert O.STREAM_TRANSITION == 0x100 and O.STREAM_EMISSION == 0x200
     assert np.allclose(x, want, rtol=0, atol=1e-12)
