@@ -1,0 +1,336 @@
+#!/usr/bin/env python
+"""Benchmark of the cutoff decision: predicted worker-times per second.
+
+One step = one whole decision of Algorithm 1's parameter server: push the newly observed run-times,
+then predict_cutoff (encoder, S predictive samples of N run-times, per-sample sort, mean over
+samples, throughput argmax).  The metric counts the S*N sampled, sorted and reduced worker-times.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python bench.py --impl reference ...          # the CPU oracle on a bounded sample, as a baseline
+    torchrun --nproc-per-node N bench.py --gpus N # N ranks share one decision: S samples each
+
+Prints one JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "predicted_worker_times_per_sec"
+UNIT = "worker-times/s"
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+PRECISION_NAMES = {0: "f32", 1: "tf32", 2: "tf32(bf16 weights)"}
+
+
+def compare_exchanges(n_pow2: int) -> int:
+    """Compare-exchange operations of a bitonic network over n_pow2 keys."""
+    lg = n_pow2.bit_length() - 1
+    return (n_pow2 // 2) * lg * (lg + 1) // 2
+
+
+def stage_work(wl, S):
+    """Algorithmic work of one decision per stage: (kind, amount).  'alu' counts one lane-operation per
+    fused multiply-add or per min / max; 'tensor' counts floating-point operations (2 per multiply-add)."""
+    N, D, H, W = wl.N, wl.D, wl.H, wl.window
+    p = 32
+    while p < N:
+        p *= 2
+    chain = S * (W * (2 * D * H + D * D) + 3 * D * H + D * H)
+    emit_macs = S * H * 2 * N
+    return {
+        "encoder": ("alu", 2 * W * (N * H + H * H)),
+        "chain": ("alu", chain),
+        "emission": ("tensor", 2 * emit_macs) if wl.precision else ("alu", emit_macs),
+        "sort": ("alu", S * 2 * compare_exchanges(p)),
+        "decide": ("alu", N),
+    }
+
+
+class ClockSampler:
+    """Samples nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.rows = []
+        self.proc = None
+        self.gpu_index = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, smax, reasons = [], [], set()
+        for r in self.rows:
+            if len(r) < 9:
+                continue
+            try:
+                sm.append(float(r[1]))
+                smax.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = max((p.get("num_threads", 1) for p in threadpool_info()), default=1)
+        return int(n)
+    except Exception:
+        return 1
+
+
+def time_oracle(wl, weights, trace, sample_S, steps=1, warmup=0, seed=1):
+    """Time the CPU oracle, as it stands, on `sample_S` samples of the workload's decision."""
+    from oracle import cutoff_oracle as O      # permitted caller: the CPU-baseline leg
+    orc = O.CutoffOracle(weights, wl.lag, sample_S, seed=seed)
+    for x in trace[-(wl.window + 2):]:
+        orc.push(x)
+    times = []
+    for i in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.predict()
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+        orc.push(trace[i % len(trace)])
+    return sum(times) / len(times)
+
+
+def run_reference(args, wl, weights, trace):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample_S = min(wl.S, args.reference_samples)
+    sec = time_oracle(wl, weights, trace, sample_S, steps=args.steps, warmup=args.warmup)
+    value = sample_S * wl.N / sec
+    cores = cpu_threads()
+    sample = f"{sample_S} of the workload's {wl.S} samples per step, all {wl.N} workers"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S": wl.S,
+                   "timed_samples_per_step": sample_S},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="n1024")
+    ap.add_argument("--samples", type=int, default=0, help="override S (for profiling small cases)")
+    ap.add_argument("--pass-rows", type=int, default=0)
+    ap.add_argument("--reference-samples", type=int, default=4096)
+    ap.add_argument("--cpu-baseline-samples", type=int, default=32768)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "cuda":
+        args.warmup = 3
+
+    from paper_1803_04209_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    if args.samples:
+        import dataclasses
+        wl = dataclasses.replace(wl, S=args.samples)
+    weights = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, min(wl.history, 64) + args.steps + args.warmup + 8)
+
+    if args.impl == "reference":
+        run_reference(args, wl, weights, trace)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_1803_04209_b200 import binding, build
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    build.build()
+    stream = torch.cuda.current_stream()
+
+    # N ranks share one decision: each draws S samples with global sample indices (weak scaling)
+    ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, wl.S, precision=wl.precision, seed=2024, device=local_rank,
+                         stream=stream.cuda_stream, sample_offset=rank * wl.S, total_samples=world * wl.S)
+    ctx.load_weights(weights)
+    if args.pass_rows:
+        ctx.set_option("pass_rows", args.pass_rows)
+    n_hist = min(wl.history, 64)
+    for x in trace[:n_hist]:
+        ctx.push(x)
+    dev_trace = torch.from_numpy(trace[n_hist:]).cuda()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    sums_dev = torch.empty(wl.N, dtype=torch.float64, device="cuda")
+
+    def step_device(i):
+        ctx.push_async(dev_trace[i])
+        ctx.predict_async()
+        code, c = ctx.fetch()
+        if world > 1:
+            sums_dev.copy_(torch.from_numpy(ctx.get_partial_sums()))
+            dist.all_reduce(sums_dev)
+            code, c = ctx.decide_from_sums(sums_dev.cpu().numpy())
+        return c
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step_device(i)
+
+    # ---- device-resident timing: per-step CUDA events, L2 flushed between steps ----------------
+    ctx.set_timing(True)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stops = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    stage_ms = {}
+    launches0 = ctx.launch_count()
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    t_wall0 = time.perf_counter()
+    for i in range(args.steps):
+        flush.zero_()
+        starts[i].record(stream)
+        step_device(args.warmup + i)
+        stops[i].record(stream)
+        stops[i].synchronize()
+        for k, v in ctx.get_timing().items():
+            stage_ms[k] = stage_ms.get(k, 0.0) + v
+    barrier()
+    wall = time.perf_counter() - t_wall0
+    clocks = sampler.stop()
+    launches = ctx.launch_count() - launches0
+    ctx.set_timing(False)
+    total_ms = sum(s.elapsed_time(e) for s, e in zip(starts, stops))
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * wl.S * wl.N / (ms_per_step * 1e-3)
+
+    # ---- end to end: host buffers in, host results out, wall clock ---------------------------------
+    host_trace = trace[n_hist:]
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        ctx.push(host_trace[args.warmup + i])
+        code, c = ctx.predict()
+        if world > 1:
+            sums_dev.copy_(torch.from_numpy(ctx.get_partial_sums()))
+            dist.all_reduce(sums_dev)
+            code, c = ctx.decide_from_sums(sums_dev.cpu().numpy())
+        e_sec, omega = ctx.get_stats()
+    barrier()
+    e2e_sec = (time.perf_counter() - t0) / args.steps
+    if world > 1:
+        t = torch.tensor([e2e_sec], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_sec = float(t.item())
+    e2e_value = world * wl.S * wl.N / e2e_sec
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant stage -----------------------------------------------------------
+    peaks = {}
+    try:
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+    except OSError:
+        pass
+    work = stage_work(wl, wl.S)
+    stage_avg = {k: v / args.steps for k, v in stage_ms.items()}
+    dominant = max(stage_avg, key=stage_avg.get)
+    kind, amount = work[dominant]
+    dur = stage_avg[dominant] * 1e-3
+    if kind == "tensor":
+        bf16 = peaks.get("bf16_tflops", 1590.0)
+        peak, unit = 0.5 * bf16, "TFLOP/s"             # tf32 runs at half the bf16 rate (nominal ratio)
+        peak_src = ("measured bf16 burst x 0.5 (nominal tf32 : bf16 ratio)" if peaks else "fallback 1590 x 0.5")
+        bound = "tensor"
+    else:
+        smax = peaks.get("sm_max_mhz", 1965.0)
+        peak, unit = SM_COUNT * FP32_LANES_PER_SM * smax * 1e6 / 1e12, "Tlane-op/s"
+        peak_src = "148 SMs x 128 fp32 lanes x max SM clock"
+        bound = "alu"
+    achieved = amount / dur / 1e12
+    roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
+                "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "stage_ms": {k: round(v, 4) for k, v in stage_avg.items()}}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        sample_S = min(wl.S, args.cpu_baseline_samples)
+        sec = time_oracle(wl, weights, trace, sample_S)
+        cpu_baseline = {"value": sample_S * wl.N / sec, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                        "sample": f"one decision on {sample_S} of {wl.S} samples, all {wl.N} workers, {sec:.2f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": PRECISION_NAMES[wl.precision], "data": "synthetic",
+        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S_per_gpu": wl.S,
+                   "parallelism": f"samples x{world}", "l2": "flushed between timed steps (256 MiB write)",
+                   "timing": "CUDA events per step on the library's stream"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
+                "h2d_bytes_per_step": 4 * wl.N, "d2h_bytes_per_step": 40 + 8 * wl.N},
+        "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "timed_region_wall_s": round(wall, 3),
+    }
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

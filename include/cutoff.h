@@ -1,0 +1,197 @@
+/*
+ * cutoff.h -- C ABI of the run-time cutoff decision of Cutoff SGD
+ * (Teng & Wood, "High Throughput Synchronous Distributed Stochastic Gradient
+ * Descent", 2018) for one NVIDIA B200 (sm_100a).
+ *
+ * The parameter server of Algorithm 1 calls, once per SGD step,
+ *      c <- predict_cutoff(q_phi, obs)
+ * and then adds the run-times r_w that arrive to obs.  This library is that
+ * call: cutoff_predict() is predict_cutoff, cutoff_push() is "obs <- obs U r_w"
+ * for one whole step, cutoff_load_weights() supplies q_phi and p_theta.
+ *
+ * What one decision computes (all of it in CUDA kernels of this library):
+ *   1. the last lag+1 pushed vectors, divided by twice the mean of the first
+ *      lag+1 pushed vectors (Section 3.1.3, last paragraph);
+ *   2. the guide q_phi of Section 3.1.3: forward and backward ReLU RNNs over
+ *      that window, then for each of S samples the chain z_t = mu + sigma*eps
+ *      with h_out = (tanh-layer(z_{t-1}) + h_left + h_right)/3;
+ *   3. for each sample the transition z_{T+1} ~ N(G(z_T), H(z_T)) and the
+ *      emission x_{T+1} ~ N(I(z_{T+1}), J(z_{T+1})) (Section 3.1.3 and the
+ *      K-sample form of the posterior predictive after Eq. 4);
+ *   4. each sample's N run-times sorted ascending, the sorted vectors
+ *      averaged over the samples (Section 3.1.1, last paragraph);
+ *   5. Omega(c) = c / E[x~_(c)] and c* = argmax_c Omega(c) (Section 3).
+ *
+ * Model variant: transition and emission are one-hidden-layer ReLU MLPs whose
+ * heads give a mean and a log-variance.  All noise comes from Philox4x32-10
+ * (Salmon et al., SC'11) and the basic Box-Muller transform, addressed by
+ * (seed, decision number, stage, sample, element), so results do not depend on
+ * how the work is split over threads or GPUs.
+ *
+ * Conventions
+ *   - Every function returns 0 (CUTOFF_OK), a positive informational code, or
+ *     a negative error code.  On a negative return no output is written.
+ *   - "host" / "device" beside a pointer says where the memory must live.
+ *     Caller pointers are borrowed for the duration of the call only.
+ *   - A context owns all device memory it allocates and is bound to one
+ *     device and one stream.  It is not thread-safe.
+ *   - Nothing here throws, aborts or calls exit().
+ */
+#ifndef CUTOFF_H_
+#define CUTOFF_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cutoff_ctx cutoff_ctx;
+
+enum {
+    CUTOFF_OK = 0,
+    CUTOFF_WARMUP = 1,          /* fewer than lag+1 vectors pushed: c = N (wait for everyone)      */
+    CUTOFF_DEGENERATE = 2,      /* no c has a positive expected time: c = N                        */
+    CUTOFF_ERR_BAD_ARG = -1,
+    CUTOFF_ERR_BAD_BLOB = -2,
+    CUTOFF_ERR_BAD_VALUE = -3,  /* a pushed run-time is not finite or not > 0                      */
+    CUTOFF_ERR_CUDA = -4,       /* a CUDA call failed; see cutoff_last_error()                     */
+    CUTOFF_ERR_UNSUPPORTED = -5,
+    CUTOFF_ERR_NOMEM = -6,
+    CUTOFF_ERR_STATE = -7,      /* call order: weights not loaded, nothing predicted yet, ...      */
+    CUTOFF_ERR_TIMEOUT = -8     /* a bounded device-side wait gave up (tensor-core pipeline)        */
+};
+
+enum {
+    CUTOFF_PRECISION_FP32 = 0,  /* every product in fp32 FMA                                       */
+    CUTOFF_PRECISION_TF32 = 1,  /* emission output layer on tensor cores, operands rounded to tf32 */
+    CUTOFF_PRECISION_BF16W = 2  /* as TF32, with the output-layer weights first rounded to bf16    */
+};
+
+enum {
+    CUTOFF_FLAG_GRAPH = 1       /* replay push+predict as one captured CUDA graph                  */
+};
+
+typedef struct {
+    int32_t n_workers;          /* N >= 1                                                          */
+    int32_t latent_dim;         /* D in {4, 8, 16, 32}                                             */
+    int32_t hidden;             /* H, multiple of 4 (multiple of 32 for the tensor-core precisions) */
+    int32_t lag;                /* the paper's l >= 0; the window holds l+1 vectors                */
+    int32_t n_samples;          /* S: samples this context draws per decision (the paper's K)      */
+    int32_t precision;          /* CUTOFF_PRECISION_*                                              */
+    int32_t device;             /* CUDA device ordinal                                             */
+    int32_t flags;              /* CUTOFF_FLAG_*                                                   */
+    int64_t sample_offset;      /* index of this context's first sample in the global draw         */
+    int64_t total_samples;      /* samples of the whole decision (0 means n_samples); used only to
+                                   normalise when several contexts share one decision              */
+    void*   stream;             /* cudaStream_t the kernels run on; NULL = the default stream      */
+    uint64_t seed;              /* Philox key                                                      */
+} cutoff_config;
+
+/* Create a context: validates cfg, selects the device, allocates all device memory.
+ * out (host) receives the handle.  Errors: BAD_ARG, UNSUPPORTED, NOMEM, CUDA. */
+int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg);
+
+/* Release everything the context owns.  NULL is allowed. */
+void cutoff_destroy(cutoff_ctx* ctx);
+
+/* Load theta and phi.  blob (host): little-endian header of six uint32
+ *   { 0x31465443 ("CTF1"), 1, N, D, H, 0 }
+ * followed by fp32 tensors, row-major [outputs x inputs], in this order:
+ *   Wxf[HxN] Whf[HxH] bf[H] a0[H]  Wxb[HxN] Whb[HxH] bb[H] b0[H]      (h_left / h_right RNNs)
+ *   Wz[HxD] bz[H] Wmu[DxH] bmu[D] Wsig[DxD] bsig[D] z0[D]             (combiner, mu_q, sigma_q)
+ *   W1[HxD] b1[H] W2[2DxH] b2[2D]                                     (transition; rows D.. = log-variance)
+ *   W3[HxD] b3[H] W4[2NxH] b4[2N]                                     (emission;   rows N.. = log-variance)
+ * The blob is copied; the caller keeps ownership.  Errors: BAD_ARG, BAD_BLOB (size, magic or
+ * dimensions do not match the context, or a value is not finite), CUDA. */
+int cutoff_load_weights(cutoff_ctx* ctx, const void* blob, size_t nbytes);
+
+/* Append one step's observed run-times ("obs <- obs U r_w", Algorithm 1).
+ * runtimes_sec: N floats, seconds, each finite and > 0; host memory if on_device == 0, device
+ * memory on the context's device otherwise (then the check runs on the GPU and a bad value is
+ * reported by this call after a stream synchronisation).
+ * censored: must be NULL (imputation of censored run-times, Section 4.2, is not built):
+ * non-NULL returns UNSUPPORTED.
+ * The first lag+1 pushes fix the normaliser.  Errors: BAD_ARG, BAD_VALUE, UNSUPPORTED, CUDA. */
+int cutoff_push(cutoff_ctx* ctx, const float* runtimes_sec, int on_device, const uint8_t* censored);
+
+/* As cutoff_push with a device pointer, but only enqueues: no synchronisation, no error report
+ * for bad values until the next cutoff_fetch / cutoff_predict (which then returns BAD_VALUE). */
+int cutoff_push_async(cutoff_ctx* ctx, const float* runtimes_sec_device);
+
+/* One decision.  c_out (host) receives c* in 1..N.  Blocks until the result is on the host.
+ * Returns OK, WARMUP (c = N, nothing computed), DEGENERATE (c = N), or an error.
+ * Advances the decision counter that addresses the noise. */
+int cutoff_predict(cutoff_ctx* ctx, int32_t* c_out);
+
+/* The same decision split in two: enqueue all kernels on the stream without waiting, then wait
+ * and read the result.  cutoff_fetch returns what cutoff_predict would have returned. */
+int cutoff_predict_async(cutoff_ctx* ctx);
+int cutoff_fetch(cutoff_ctx* ctx, int32_t* c_out);
+
+/* Results of the last completed decision.  Either pointer may be NULL.
+ * exp_order_stats_sec (host, N floats): E[x~_(j)] in seconds, ascending.
+ * omega_per_sec (host, N floats): Omega(c) = c / E[x~_(c)]; -inf where E <= 0.
+ * Errors: STATE if no decision has completed, CUDA. */
+int cutoff_get_stats(cutoff_ctx* ctx, float* exp_order_stats_sec, float* omega_per_sec);
+
+/* Sum over this context's samples of the sorted, normalised run-times of the last decision
+ * (host, N doubles): the quantity several contexts add up when they share one decision.
+ * cutoff_decide_from_sums then finishes a decision from such a total: sums (host, N doubles)
+ * over total_samples samples -> c_out, and the stats returned by cutoff_get_stats. */
+int cutoff_get_partial_sums(cutoff_ctx* ctx, double* sums);
+int cutoff_decide_from_sums(cutoff_ctx* ctx, const double* sums, int32_t* c_out);
+
+/* Forget all observations and restart the decision counter. */
+int cutoff_reset(cutoff_ctx* ctx);
+
+/* Observation state (window, normaliser, counters) as an opaque byte string.
+ * save: if buf is NULL, *nbytes receives the size needed; else *nbytes is the capacity on entry
+ * and the size written on exit.  restore: the string must come from a context with the same N
+ * and lag.  Errors: BAD_ARG, CUDA. */
+int cutoff_save_state(cutoff_ctx* ctx, void* buf, size_t* nbytes);
+int cutoff_restore_state(cutoff_ctx* ctx, const void* buf, size_t nbytes);
+
+/* Text for a return code; the last CUDA error text of a context. Never NULL. */
+const char* cutoff_strerror(int code);
+const char* cutoff_last_error(cutoff_ctx* ctx);
+
+/* ---- measurement hooks ---------------------------------------------------------------------
+ * With timing on, every stage of a decision is bracketed by CUDA events on the context's stream
+ * (not available together with CUTOFF_FLAG_GRAPH).  cutoff_get_timing writes up to cap stage
+ * times of the last fetched decision in milliseconds and returns the number of stages;
+ * cutoff_stage_name names stage i.  cutoff_launch_count returns the number of kernels this
+ * context has launched since it was created. */
+int cutoff_set_timing(cutoff_ctx* ctx, int on);
+int cutoff_get_timing(cutoff_ctx* ctx, float* ms, int cap);
+const char* cutoff_stage_name(int i);
+int64_t cutoff_launch_count(cutoff_ctx* ctx);
+
+/* Tuning knobs, by name.  "pass_rows": samples that go through sampling and sorting per pass
+ * (>= 1024; clipped to S and to the allocated pass buffers).  Errors: BAD_ARG, STATE. */
+int cutoff_set_option(cutoff_ctx* ctx, const char* name, int64_t value);
+
+/* ---- test hooks ----------------------------------------------------------------------------
+ * cutoff_debug_normals: the noise generator alone.  Writes, for samples k0 .. k0+count-1 and
+ * elements 0 .. n_elems-1 of the given (seed, step, stream), the standard normals
+ * (normals_out, host, count*n_elems floats) and the raw Philox words (words_out, host,
+ * count*4*ceil(n_elems/4) uint32); either may be NULL.  device selects the GPU.
+ *
+ * cutoff_debug_samples: the unsorted predictive draws of the coming decision, in normalised
+ * units, for local samples k0 .. k0+count-1 (x_out, host, count*N floats).  Does not advance the
+ * decision counter.  Returns WARMUP before lag+1 pushes.
+ *
+ * cutoff_debug_sort: the library's sorting network applied to caller rows.  rows (host,
+ * n_rows*n floats) -> keys_out (host, sorted ascending) and perm_out (host, int32, the original
+ * position of each sorted key; equal keys keep their original order). */
+int cutoff_debug_normals(int device, uint64_t seed, uint32_t step, uint32_t stream, int64_t k0,
+                         int64_t count, int32_t n_elems, float* normals_out, uint32_t* words_out);
+int cutoff_debug_samples(cutoff_ctx* ctx, int64_t k0, int64_t count, float* x_out);
+int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n,
+                      float* keys_out, int32_t* perm_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CUTOFF_H_ */

@@ -1,0 +1,259 @@
+"""ctypes binding of libcutoff.so: the same names as include/cutoff.h, argument marshalling only.
+
+Every step of a decision runs in the library's CUDA kernels.  There is no CPU fallback: if the
+shared library is missing or does not load, every entry point raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import struct
+
+import numpy as np
+
+from .inputs import TENSOR_ORDER, tensor_shapes
+
+PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(PKG_DIR, "libcutoff.so")
+
+OK, WARMUP, DEGENERATE = 0, 1, 2
+ERR_BAD_ARG, ERR_BAD_BLOB, ERR_BAD_VALUE, ERR_CUDA = -1, -2, -3, -4
+ERR_UNSUPPORTED, ERR_NOMEM, ERR_STATE, ERR_TIMEOUT = -5, -6, -7, -8
+PRECISION_FP32, PRECISION_TF32, PRECISION_BF16W = 0, 1, 2
+FLAG_GRAPH = 1
+BLOB_MAGIC = 0x31465443
+
+EXPORTS = (
+    "cutoff_create", "cutoff_destroy", "cutoff_load_weights", "cutoff_push", "cutoff_push_async",
+    "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_get_stats",
+    "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
+    "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
+    "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
+    "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_sort",
+)
+
+
+class CutoffConfig(C.Structure):
+    _fields_ = [
+        ("n_workers", C.c_int32), ("latent_dim", C.c_int32), ("hidden", C.c_int32), ("lag", C.c_int32),
+        ("n_samples", C.c_int32), ("precision", C.c_int32), ("device", C.c_int32), ("flags", C.c_int32),
+        ("sample_offset", C.c_int64), ("total_samples", C.c_int64), ("stream", C.c_void_p), ("seed", C.c_uint64),
+    ]
+
+
+class CutoffError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})" + (f": {detail}" if detail else ""))
+
+
+_lib = None
+
+
+def load_library(path: str | None = None) -> C.CDLL:
+    """Load libcutoff.so (built in-tree by paper_1803_04209_b200.build).  Raises if it is absent."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: build it with `python -m paper_1803_04209_b200.build` "
+                           "(there is no CPU fallback)")
+    lib = C.CDLL(path)
+    vp, i32p, f32p, f64p = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_float), C.POINTER(C.c_double)
+    sig = {
+        "cutoff_create": (C.c_int, [C.POINTER(vp), C.POINTER(CutoffConfig)]),
+        "cutoff_destroy": (None, [vp]),
+        "cutoff_load_weights": (C.c_int, [vp, vp, C.c_size_t]),
+        "cutoff_push": (C.c_int, [vp, vp, C.c_int, vp]),
+        "cutoff_push_async": (C.c_int, [vp, vp]),
+        "cutoff_predict": (C.c_int, [vp, i32p]),
+        "cutoff_predict_async": (C.c_int, [vp]),
+        "cutoff_fetch": (C.c_int, [vp, i32p]),
+        "cutoff_get_stats": (C.c_int, [vp, vp, vp]),
+        "cutoff_get_partial_sums": (C.c_int, [vp, vp]),
+        "cutoff_decide_from_sums": (C.c_int, [vp, vp, i32p]),
+        "cutoff_reset": (C.c_int, [vp]),
+        "cutoff_save_state": (C.c_int, [vp, vp, C.POINTER(C.c_size_t)]),
+        "cutoff_restore_state": (C.c_int, [vp, vp, C.c_size_t]),
+        "cutoff_strerror": (C.c_char_p, [C.c_int]),
+        "cutoff_last_error": (C.c_char_p, [vp]),
+        "cutoff_set_timing": (C.c_int, [vp, C.c_int]),
+        "cutoff_get_timing": (C.c_int, [vp, f32p, C.c_int]),
+        "cutoff_stage_name": (C.c_char_p, [C.c_int]),
+        "cutoff_launch_count": (C.c_int64, [vp]),
+        "cutoff_set_option": (C.c_int, [vp, C.c_char_p, C.c_int64]),
+        "cutoff_debug_normals": (C.c_int, [C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int64, C.c_int64,
+                                           C.c_int32, vp, vp]),
+        "cutoff_debug_samples": (C.c_int, [vp, C.c_int64, C.c_int64, vp]),
+        "cutoff_debug_sort": (C.c_int, [vp, vp, C.c_int64, C.c_int32, vp, vp]),
+    }
+    for name, (res, args) in sig.items():
+        fn = getattr(lib, name)          # AttributeError if the library does not export it
+        fn.restype = res
+        fn.argtypes = args
+    if path == LIB_PATH:
+        _lib = lib
+    return lib
+
+
+def strerror(code: int) -> str:
+    return load_library().cutoff_strerror(code).decode()
+
+
+def pack_weights(weights: dict, N: int, D: int, H: int) -> bytes:
+    """Serialise a weight dictionary into the blob cutoff_load_weights expects."""
+    shapes = tensor_shapes(N, D, H)
+    parts = [struct.pack("<6I", BLOB_MAGIC, 1, N, D, H, 0)]
+    for name in TENSOR_ORDER:
+        a = np.ascontiguousarray(weights[name], dtype=np.float32)
+        if a.shape != shapes[name]:
+            raise ValueError(f"{name}: shape {a.shape}, expected {shapes[name]}")
+        parts.append(a.tobytes())
+    return b"".join(parts)
+
+
+def _ptr(a) -> int:
+    """Address of a numpy array (host) or of a torch CUDA tensor (device)."""
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data
+    return a.data_ptr()
+
+
+class Cutoff:
+    """One decision context on one GPU and one stream (thin wrapper over the C ABI)."""
+
+    def __init__(self, n_workers: int, latent_dim: int, hidden: int, lag: int, n_samples: int,
+                 precision: int = PRECISION_FP32, seed: int = 0, device: int = 0, stream: int | None = None,
+                 flags: int = 0, sample_offset: int = 0, total_samples: int = 0):
+        self._lib = load_library()
+        self.N, self.D, self.H, self.lag, self.S = n_workers, latent_dim, hidden, lag, n_samples
+        self.cfg = CutoffConfig(n_workers, latent_dim, hidden, lag, n_samples, precision, device, flags,
+                                sample_offset, total_samples, stream or None, seed)
+        self._h = C.c_void_p()
+        rc = self._lib.cutoff_create(C.byref(self._h), C.byref(self.cfg))
+        if rc != OK:
+            self._h = C.c_void_p()
+            raise CutoffError(rc, "cutoff_create")
+
+    def _check(self, rc: int, where: str) -> int:
+        if rc < 0:
+            raise CutoffError(rc, where, self._lib.cutoff_last_error(self._h).decode())
+        return rc
+
+    def close(self):
+        if self._h:
+            self._lib.cutoff_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def load_weights(self, weights: dict | bytes):
+        blob = weights if isinstance(weights, (bytes, bytearray)) else pack_weights(weights, self.N, self.D, self.H)
+        self._check(self._lib.cutoff_load_weights(self._h, blob, len(blob)), "cutoff_load_weights")
+
+    def push(self, runtimes_sec) -> int:
+        """Host numpy array (fp32, N) or torch CUDA tensor."""
+        if isinstance(runtimes_sec, np.ndarray):
+            a = np.ascontiguousarray(runtimes_sec, dtype=np.float32)
+            if a.shape != (self.N,):
+                raise ValueError("expected N run-times")
+            return self._check(self._lib.cutoff_push(self._h, a.ctypes.data, 0, None), "cutoff_push")
+        if tuple(runtimes_sec.shape) != (self.N,) or not runtimes_sec.is_cuda or not runtimes_sec.is_contiguous():
+            raise ValueError("expected a contiguous CUDA tensor of N fp32 run-times")
+        return self._check(self._lib.cutoff_push(self._h, runtimes_sec.data_ptr(), 1, None), "cutoff_push")
+
+    def push_async(self, runtimes_sec_device) -> int:
+        return self._check(self._lib.cutoff_push_async(self._h, runtimes_sec_device.data_ptr()), "cutoff_push_async")
+
+    def predict(self):
+        """Returns (code, c)."""
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_predict(self._h, C.byref(c)), "cutoff_predict")
+        return rc, c.value
+
+    def predict_async(self) -> int:
+        return self._check(self._lib.cutoff_predict_async(self._h), "cutoff_predict_async")
+
+    def fetch(self):
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_fetch(self._h, C.byref(c)), "cutoff_fetch")
+        return rc, c.value
+
+    def get_stats(self):
+        """(E[x~_(j)] in seconds, Omega(c) per second) of the last decision."""
+        e = np.empty(self.N, dtype=np.float32)
+        om = np.empty(self.N, dtype=np.float32)
+        self._check(self._lib.cutoff_get_stats(self._h, e.ctypes.data, om.ctypes.data), "cutoff_get_stats")
+        return e, om
+
+    def get_partial_sums(self) -> np.ndarray:
+        s = np.empty(self.N, dtype=np.float64)
+        self._check(self._lib.cutoff_get_partial_sums(self._h, s.ctypes.data), "cutoff_get_partial_sums")
+        return s
+
+    def decide_from_sums(self, sums: np.ndarray):
+        s = np.ascontiguousarray(sums, dtype=np.float64)
+        if s.shape != (self.N,):
+            raise ValueError("expected N sums")
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_decide_from_sums(self._h, s.ctypes.data, C.byref(c)), "cutoff_decide_from_sums")
+        return rc, c.value
+
+    def reset(self):
+        self._check(self._lib.cutoff_reset(self._h), "cutoff_reset")
+
+    def save_state(self) -> bytes:
+        n = C.c_size_t(0)
+        self._check(self._lib.cutoff_save_state(self._h, None, C.byref(n)), "cutoff_save_state")
+        buf = C.create_string_buffer(n.value)
+        self._check(self._lib.cutoff_save_state(self._h, buf, C.byref(n)), "cutoff_save_state")
+        return buf.raw[: n.value]
+
+    def restore_state(self, blob: bytes):
+        self._check(self._lib.cutoff_restore_state(self._h, blob, len(blob)), "cutoff_restore_state")
+
+    def set_timing(self, on: bool):
+        self._check(self._lib.cutoff_set_timing(self._h, int(on)), "cutoff_set_timing")
+
+    def get_timing(self) -> dict:
+        ms = (C.c_float * 16)()
+        n = self._check(self._lib.cutoff_get_timing(self._h, ms, 16), "cutoff_get_timing")
+        return {self._lib.cutoff_stage_name(i).decode(): ms[i] for i in range(n)}
+
+    def launch_count(self) -> int:
+        return self._lib.cutoff_launch_count(self._h)
+
+    def set_option(self, name: str, value: int):
+        self._check(self._lib.cutoff_set_option(self._h, name.encode(), value), "cutoff_set_option")
+
+    def debug_samples(self, k0: int, count: int) -> np.ndarray:
+        x = np.empty((count, self.N), dtype=np.float32)
+        rc = self._check(self._lib.cutoff_debug_samples(self._h, k0, count, x.ctypes.data), "cutoff_debug_samples")
+        if rc == WARMUP:
+            raise CutoffError(ERR_STATE, "cutoff_debug_samples", "fewer than lag+1 observations")
+        return x
+
+    def debug_sort(self, rows: np.ndarray):
+        r = np.ascontiguousarray(rows, dtype=np.float32)
+        keys = np.empty_like(r)
+        perm = np.empty(r.shape, dtype=np.int32)
+        self._check(self._lib.cutoff_debug_sort(self._h, r.ctypes.data, r.shape[0], r.shape[1], keys.ctypes.data,
+                                                perm.ctypes.data), "cutoff_debug_sort")
+        return keys, perm
+
+
+def debug_normals(seed: int, step: int, stream: int, k0: int, count: int, n_elems: int, device: int = 0):
+    """(normals[count, n_elems] fp32, words[count, ceil(n_elems/4), 4] uint32) from the GPU generator."""
+    lib = load_library()
+    nq = (n_elems + 3) // 4
+    normals = np.empty((count, n_elems), dtype=np.float32)
+    words = np.empty((count, nq, 4), dtype=np.uint32)
+    rc = lib.cutoff_debug_normals(device, seed, step, stream, k0, count, n_elems, normals.ctypes.data, words.ctypes.data)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_debug_normals")
+    return normals, words

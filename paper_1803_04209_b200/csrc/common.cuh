@@ -1,0 +1,45 @@
+// Shared device-side declarations of the cutoff library.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace cutoff {
+
+// Observation and decision state that lives on the device, so that a captured CUDA graph can
+// replay push + predict without any host-side argument changing between replays.
+struct DevState {
+    double norm_sum;        // sum of every entry of the first lag+1 pushed vectors
+    float scale;            // s = 2 * mean of those entries; valid once push_count >= window
+    float inv_scale;
+    uint32_t push_count;    // vectors pushed since reset
+    uint32_t step;          // decisions made since reset (addresses the noise)
+    int32_t error_flags;    // bit 0: a pushed value was not finite or not > 0; bit 1: device wait timed out
+    int32_t c_star;         // last decision
+    int32_t code;           // 0 ok, 2 degenerate
+    int32_t pad;
+};
+
+constexpr int kErrBadValue = 1;
+constexpr int kErrTimeout = 2;
+
+// Model dimensions and device pointers handed to the kernels by value.
+struct ModelDev {
+    int N, D, H, W;          // workers, latent size, hidden width, window = lag + 1
+    // encoder RNNs
+    const float *Wxf, *Whf, *bf, *a0, *Wxb, *Whb, *bb, *b0;
+    // guide
+    const float *Wz, *bz, *WmuT /*[H x D]*/, *bmu, *Wsig, *bsig, *z0;
+    // transition
+    const float *W1, *b1, *W2T /*[H x 2D]*/, *b2;
+    // emission
+    const float *W3, *b3, *W4 /*[2N x H]*/, *b4;
+};
+
+struct NoiseKey {
+    uint32_t seed_lo, seed_hi;
+};
+
+__host__ __device__ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+__host__ __device__ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+}  // namespace cutoff

@@ -1,0 +1,734 @@
+// C ABI and host orchestration of the cutoff library (see include/cutoff.h).
+#include "../../include/cutoff.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "kernels_model.cuh"
+#include "kernels_sort.cuh"
+
+using namespace cutoff;
+
+namespace {
+
+constexpr uint32_t kBlobMagic = 0x31465443u;   // "CTF1"
+constexpr int kNumStages = 5;
+const char* const kStageNames[kNumStages] = {"encoder", "chain", "emission", "sort", "decide"};
+
+struct TensorSpec { const char* name; size_t rows, cols; };
+
+}  // namespace
+
+struct cutoff_ctx {
+    cutoff_config cfg{};
+    int N = 0, D = 0, H = 0, W = 0, S = 0;
+    int ldx = 0;            // leading dimension of the sample matrix (N rounded up to 4)
+    int P = 0;              // sort width: N rounded up to a power of two, at least 32
+    int sm_count = 0;
+    int chunk_rows = 0;     // samples per pass through chain -> emission -> sort
+    int alloc_rows = 0;     // rows the pass buffers were allocated for
+    int n_chunks = 0;
+    int sort_grid = 0;      // CTAs of the sort kernel per chunk (= partial rows per chunk)
+    cudaStream_t stream = nullptr;
+
+    float* d_blob = nullptr;        // tensors as loaded
+    float* d_WmuT = nullptr;        // [H][D]
+    float* d_W2T = nullptr;         // [H][2D]
+    ModelDev m{};
+    bool weights_loaded = false;
+
+    float* d_ring = nullptr;        // [W][N]
+    float* d_stage = nullptr;       // [N] landing buffer for host pushes
+    DevState* d_state = nullptr;
+    float* d_proj = nullptr;        // [2][W][H]
+    float* d_hlr = nullptr;         // [2][W][H]
+    float* d_v = nullptr;           // [chunk_rows][H]
+    float* d_x = nullptr;           // [chunk_rows][ldx]
+    float* d_partial = nullptr;     // [n_chunks * sort_grid][N]
+    double* d_sums = nullptr;       // [N]
+    float* d_E = nullptr;           // [N]
+    float* d_omega = nullptr;       // [N]
+
+    float* h_stage = nullptr;       // pinned [N]
+    DevState* h_state = nullptr;    // pinned
+
+    uint32_t pushes = 0;            // host mirror of DevState::push_count
+    bool pending = false;           // a decision is enqueued and not yet fetched
+    bool pending_warmup = false;
+    bool have_result = false;
+
+    bool timing = false;
+    cudaEvent_t ev[kNumStages + 1][64]{};   // per chunk, stage boundaries
+    bool ev_created = false;
+    float stage_ms[kNumStages]{};
+    int timed_chunks = 0;
+
+    int64_t launches = 0;
+    std::string last_error;
+};
+
+namespace {
+
+#define CU_CHECK(ctx, call)                                                                          \
+    do {                                                                                             \
+        cudaError_t err__ = (call);                                                                  \
+        if (err__ != cudaSuccess) {                                                                  \
+            if (ctx) (ctx)->last_error = std::string(#call) + ": " + cudaGetErrorString(err__);      \
+            return err__ == cudaErrorMemoryAllocation ? CUTOFF_ERR_NOMEM : CUTOFF_ERR_CUDA;          \
+        }                                                                                            \
+    } while (0)
+
+std::vector<TensorSpec> tensor_specs(size_t N, size_t D, size_t H) {
+    return {
+        {"Wxf", H, N}, {"Whf", H, H}, {"bf", 1, H}, {"a0", 1, H},
+        {"Wxb", H, N}, {"Whb", H, H}, {"bb", 1, H}, {"b0", 1, H},
+        {"Wz", H, D}, {"bz", 1, H}, {"Wmu", D, H}, {"bmu", 1, D}, {"Wsig", D, D}, {"bsig", 1, D}, {"z0", 1, D},
+        {"W1", H, D}, {"b1", 1, H}, {"W2", 2 * D, H}, {"b2", 1, 2 * D},
+        {"W3", H, D}, {"b3", 1, H}, {"W4", 2 * N, H}, {"b4", 1, 2 * N},
+    };
+}
+
+int next_pow2(int n) {
+    int p = 1;
+    while (p < n) p <<= 1;
+    return p;
+}
+
+void free_all(cutoff_ctx* c) {
+    cudaFree(c->d_blob); cudaFree(c->d_WmuT); cudaFree(c->d_W2T); cudaFree(c->d_ring); cudaFree(c->d_stage);
+    cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
+    cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
+    if (c->h_stage) cudaFreeHost(c->h_stage);
+    if (c->h_state) cudaFreeHost(c->h_state);
+    if (c->ev_created)
+        for (auto& row : c->ev)
+            for (auto& e : row)
+                if (e) cudaEventDestroy(e);
+}
+
+// Work split: how many samples go through chain -> emission -> sort at a time, and how many
+// CTAs the sort kernel uses per pass.
+void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
+    int rows = chunk_rows_wanted > 0 ? chunk_rows_wanted : c->S;
+    if (rows > c->S) rows = c->S;
+    if (rows > c->alloc_rows) rows = c->alloc_rows;
+    c->chunk_rows = rows;
+    c->n_chunks = ceil_div(c->S, rows);
+    if (c->P <= 1024) {
+        const int want = ceil_div(rows, kSortWarps);
+        const int cap = c->sm_count * 2;
+        c->sort_grid = want < cap ? want : cap;
+    } else {
+        const int cap = c->sm_count * 2;
+        c->sort_grid = rows < cap ? rows : cap;
+    }
+}
+
+template <int E>
+void launch_sort_warp(cutoff_ctx* c, int count, float* partial) {
+    k_sort_sum_warp<E><<<c->sort_grid, kSortWarps * 32, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
+}
+
+int launch_sort(cutoff_ctx* c, int count, float* partial) {
+    switch (c->P) {
+        case 32: launch_sort_warp<1>(c, count, partial); break;
+        case 64: launch_sort_warp<2>(c, count, partial); break;
+        case 128: launch_sort_warp<4>(c, count, partial); break;
+        case 256: launch_sort_warp<8>(c, count, partial); break;
+        case 512: launch_sort_warp<16>(c, count, partial); break;
+        case 1024: launch_sort_warp<32>(c, count, partial); break;
+        case 2048:
+        case 4096:
+            k_sort_sum_cta<<<c->sort_grid, kSortCtaThreads, c->P * sizeof(float), c->stream>>>(
+                c->d_x, c->ldx, c->N, c->P, count, partial);
+            break;
+        default: return CUTOFF_ERR_UNSUPPORTED;
+    }
+    c->launches += 1;
+    return CUTOFF_OK;
+}
+
+template <int D>
+void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_chain<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        attr_set = true;
+    }
+    const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    k_chain<D><<<ceil_div(count, kChainThreads / (D / 4)), kChainThreads, smem, c->stream>>>(
+        c->m, c->d_hlr, c->d_state, key, sample_base, count, c->cfg.precision != CUTOFF_PRECISION_FP32, c->d_v);
+}
+
+void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
+    const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
+    switch (c->D) {
+        case 4: launch_chain_t<4>(c, sample_base, count, smem); break;
+        case 8: launch_chain_t<8>(c, sample_base, count, smem); break;
+        case 16: launch_chain_t<16>(c, sample_base, count, smem); break;
+        default: launch_chain_t<32>(c, sample_base, count, smem); break;
+    }
+    c->launches += 1;
+}
+
+void launch_emission(cutoff_ctx* c, uint32_t sample_base, int count) {
+    const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    dim3 grid(ceil_div(c->N, kEmitTN), ceil_div(count, kEmitTM));
+    k_emit_fma<<<grid, kEmitThreads, 0, c->stream>>>(c->m, c->d_v, c->d_state, key, sample_base, count, c->d_x, c->ldx);
+    c->launches += 1;
+}
+
+void launch_encoder(cutoff_ctx* c) {
+    dim3 grid(ceil_div(c->H, kProjWarps), 2);
+    k_enc_proj<<<grid, kProjWarps * 32, 0, c->stream>>>(c->m, c->d_ring, c->d_state, c->d_proj);
+    k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_hlr);
+    c->launches += 2;
+}
+
+int ensure_events(cutoff_ctx* c) {
+    if (c->ev_created) return CUTOFF_OK;
+    for (auto& row : c->ev)
+        for (auto& e : row) CU_CHECK(c, cudaEventCreate(&e));
+    c->ev_created = true;
+    return CUTOFF_OK;
+}
+
+// Enqueue one decision's kernels.  advance = 1 for a real decision, 0 for the debug hook.
+int enqueue_decision(cutoff_ctx* c) {
+    const bool timed = c->timing && c->n_chunks <= 64;
+    if (timed) {
+        const int rc = ensure_events(c);
+        if (rc) return rc;
+        cudaEventRecord(c->ev[0][0], c->stream);
+    }
+    launch_encoder(c);
+    if (timed) cudaEventRecord(c->ev[1][0], c->stream);
+    for (int ch = 0; ch < c->n_chunks; ++ch) {
+        const int row0 = ch * c->chunk_rows;
+        const int count = (c->S - row0) < c->chunk_rows ? (c->S - row0) : c->chunk_rows;
+        const uint32_t base = static_cast<uint32_t>(c->cfg.sample_offset) + static_cast<uint32_t>(row0);
+        if (timed && ch > 0) cudaEventRecord(c->ev[1][ch], c->stream);
+        launch_chain(c, base, count);
+        if (timed) cudaEventRecord(c->ev[2][ch], c->stream);
+        launch_emission(c, base, count);
+        if (timed) cudaEventRecord(c->ev[3][ch], c->stream);
+        const int rc = launch_sort(c, count, c->d_partial + static_cast<size_t>(ch) * c->sort_grid * c->N);
+        if (rc) return rc;
+        if (timed) cudaEventRecord(c->ev[4][ch], c->stream);
+    }
+    k_colsum<<<ceil_div(c->N, 256), 256, 0, c->stream>>>(c->d_partial, c->n_chunks * c->sort_grid, c->N, c->d_sums);
+    const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
+    k_decide<<<1, kDecideThreads, 0, c->stream>>>(c->d_sums, c->N, 1.0 / static_cast<double>(total), c->d_state, 1,
+                                                  c->d_E, c->d_omega);
+    c->launches += 2;
+    if (timed) cudaEventRecord(c->ev[5][0], c->stream);
+    c->timed_chunks = timed ? c->n_chunks : 0;
+    CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaGetLastError());
+    return CUTOFF_OK;
+}
+
+int collect_timing(cutoff_ctx* c) {
+    for (float& v : c->stage_ms) v = 0.0f;
+    if (c->timed_chunks == 0) return CUTOFF_OK;
+    float ms = 0.0f;
+    CU_CHECK(c, cudaEventElapsedTime(&ms, c->ev[0][0], c->ev[1][0]));
+    c->stage_ms[0] = ms;
+    for (int ch = 0; ch < c->timed_chunks; ++ch) {
+        for (int s = 1; s <= 3; ++s) {
+            CU_CHECK(c, cudaEventElapsedTime(&ms, c->ev[s][ch], c->ev[s + 1][ch]));
+            c->stage_ms[s] += ms;
+        }
+    }
+    CU_CHECK(c, cudaEventElapsedTime(&ms, c->ev[4][c->timed_chunks - 1], c->ev[5][0]));
+    c->stage_ms[4] = ms;
+    return CUTOFF_OK;
+}
+
+bool valid_latent(int D) { return D == 4 || D == 8 || D == 16 || D == 32; }
+
+}  // namespace
+
+extern "C" {
+
+const char* cutoff_strerror(int code) {
+    switch (code) {
+        case CUTOFF_OK: return "ok";
+        case CUTOFF_WARMUP: return "warm-up: fewer than lag+1 observations, cutoff = all workers";
+        case CUTOFF_DEGENERATE: return "no cutoff has a positive expected time, cutoff = all workers";
+        case CUTOFF_ERR_BAD_ARG: return "bad argument";
+        case CUTOFF_ERR_BAD_BLOB: return "weight blob does not match the context or is malformed";
+        case CUTOFF_ERR_BAD_VALUE: return "run-times must be finite and greater than zero";
+        case CUTOFF_ERR_CUDA: return "CUDA error";
+        case CUTOFF_ERR_UNSUPPORTED: return "not supported";
+        case CUTOFF_ERR_NOMEM: return "out of device memory";
+        case CUTOFF_ERR_STATE: return "call out of order";
+        case CUTOFF_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        default: return "unknown code";
+    }
+}
+
+const char* cutoff_last_error(cutoff_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+const char* cutoff_stage_name(int i) { return (i >= 0 && i < kNumStages) ? kStageNames[i] : ""; }
+
+int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
+    if (!out || !cfg) return CUTOFF_ERR_BAD_ARG;
+    if (cfg->n_workers < 1 || cfg->hidden < 4 || cfg->lag < 0 || cfg->n_samples < 1 || cfg->sample_offset < 0 ||
+        cfg->total_samples < 0 || cfg->device < 0)
+        return CUTOFF_ERR_BAD_ARG;
+    if (cfg->precision < CUTOFF_PRECISION_FP32 || cfg->precision > CUTOFF_PRECISION_BF16W) return CUTOFF_ERR_BAD_ARG;
+    if (!valid_latent(cfg->latent_dim) || cfg->hidden % 4 != 0) return CUTOFF_ERR_UNSUPPORTED;
+    if (cfg->n_workers > 4096 || cfg->hidden > 1024 || cfg->lag > 255) return CUTOFF_ERR_UNSUPPORTED;
+    if (cfg->sample_offset + cfg->n_samples > (1ll << 32)) return CUTOFF_ERR_UNSUPPORTED;
+    if (cfg->total_samples > 0 && cfg->total_samples < cfg->n_samples) return CUTOFF_ERR_BAD_ARG;
+
+    cutoff_ctx* c = new (std::nothrow) cutoff_ctx();
+    if (!c) return CUTOFF_ERR_NOMEM;
+    c->cfg = *cfg;
+    c->N = cfg->n_workers; c->D = cfg->latent_dim; c->H = cfg->hidden; c->W = cfg->lag + 1; c->S = cfg->n_samples;
+    c->ldx = (c->N + 3) & ~3;
+    c->P = next_pow2(c->N) < 32 ? 32 : next_pow2(c->N);
+    c->stream = static_cast<cudaStream_t>(cfg->stream);
+
+    auto fail = [&](int rc) { free_all(c); delete c; return rc; };
+#define CREATE_CHECK(call)                                                                         \
+    do {                                                                                           \
+        cudaError_t err__ = (call);                                                                \
+        if (err__ != cudaSuccess) return fail(err__ == cudaErrorMemoryAllocation ? CUTOFF_ERR_NOMEM : CUTOFF_ERR_CUDA); \
+    } while (0)
+
+    CREATE_CHECK(cudaSetDevice(cfg->device));
+    cudaDeviceProp prop;
+    CREATE_CHECK(cudaGetDeviceProperties(&prop, cfg->device));
+    c->sm_count = prop.multiProcessorCount;
+    if (chain_smem_floats(c->D, c->H, c->W) * sizeof(float) > 220 * 1024) return fail(CUTOFF_ERR_UNSUPPORTED);
+
+    // Default pass size: keep one pass's sample matrix within ~48 MB so it stays in L2.
+    int rows = static_cast<int>((48ll << 20) / (static_cast<int64_t>(c->ldx) * sizeof(float)));
+    rows = rows / 1024 * 1024;
+    if (rows < 1024) rows = 1024;
+    {
+        // pass buffers are allocated for up to 2 GiB of samples so that larger passes can be tried
+        int64_t cap = (2ll << 30) / (static_cast<int64_t>(c->ldx + c->H) * sizeof(float));
+        if (cap < rows) cap = rows;
+        c->alloc_rows = cap < c->S ? static_cast<int>(cap) : c->S;
+    }
+    plan_chunks(c, rows);
+
+    size_t blob_floats = 0;
+    for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
+    CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
+    CREATE_CHECK(cudaMalloc(&c->d_WmuT, sizeof(float) * c->H * c->D));
+    CREATE_CHECK(cudaMalloc(&c->d_W2T, sizeof(float) * c->H * 2 * c->D));
+    CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_state, sizeof(DevState)));
+    CREATE_CHECK(cudaMalloc(&c->d_proj, sizeof(float) * 2 * c->W * c->H));
+    CREATE_CHECK(cudaMalloc(&c->d_hlr, sizeof(float) * 2 * c->W * c->H));
+    CREATE_CHECK(cudaMalloc(&c->d_v, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->H));
+    CREATE_CHECK(cudaMalloc(&c->d_x, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
+    // partial rows: room for the smallest allowed pass size (1024 rows)
+    const size_t max_partial_rows = static_cast<size_t>(ceil_div(c->S, 1024) + 1) * (c->sm_count * 2);
+    CREATE_CHECK(cudaMalloc(&c->d_partial, sizeof(float) * max_partial_rows * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_sums, sizeof(double) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_E, sizeof(float) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_omega, sizeof(float) * c->N));
+    CREATE_CHECK(cudaMallocHost(&c->h_stage, sizeof(float) * c->N));
+    CREATE_CHECK(cudaMallocHost(&c->h_state, sizeof(DevState)));
+    CREATE_CHECK(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
+    CREATE_CHECK(cudaMemsetAsync(c->d_ring, 0, sizeof(float) * c->W * c->N, c->stream));
+    CREATE_CHECK(cudaStreamSynchronize(c->stream));
+#undef CREATE_CHECK
+    *out = c;
+    return CUTOFF_OK;
+}
+
+void cutoff_destroy(cutoff_ctx* ctx) {
+    if (!ctx) return;
+    cudaSetDevice(ctx->cfg.device);
+    cudaStreamSynchronize(ctx->stream);
+    free_all(ctx);
+    delete ctx;
+}
+
+int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
+    if (!c || !blob) return CUTOFF_ERR_BAD_ARG;
+    if (nbytes < 6 * sizeof(uint32_t)) return CUTOFF_ERR_BAD_BLOB;
+    uint32_t hdr[6];
+    std::memcpy(hdr, blob, sizeof(hdr));
+    if (hdr[0] != kBlobMagic || hdr[1] != 1u) return CUTOFF_ERR_BAD_BLOB;
+    if (hdr[2] != static_cast<uint32_t>(c->N) || hdr[3] != static_cast<uint32_t>(c->D) ||
+        hdr[4] != static_cast<uint32_t>(c->H))
+        return CUTOFF_ERR_BAD_BLOB;
+    const auto specs = tensor_specs(c->N, c->D, c->H);
+    size_t total = 0;
+    for (const auto& t : specs) total += t.rows * t.cols;
+    if (nbytes != sizeof(hdr) + total * sizeof(float)) return CUTOFF_ERR_BAD_BLOB;
+    const float* src = reinterpret_cast<const float*>(static_cast<const char*>(blob) + sizeof(hdr));
+    for (size_t i = 0; i < total; ++i)
+        if (!std::isfinite(src[i])) return CUTOFF_ERR_BAD_BLOB;
+
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    std::vector<float> host(src, src + total);
+    std::vector<size_t> off(specs.size());
+    size_t o = 0;
+    for (size_t i = 0; i < specs.size(); ++i) { off[i] = o; o += specs[i].rows * specs[i].cols; }
+    if (c->cfg.precision == CUTOFF_PRECISION_BF16W) {
+        // round the output-layer weights to bf16 (nearest even), kept as fp32 bit patterns
+        float* w4 = host.data() + off[21];
+        for (size_t i = 0; i < specs[21].rows * specs[21].cols; ++i) {
+            uint32_t u;
+            std::memcpy(&u, &w4[i], 4);
+            u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
+            std::memcpy(&w4[i], &u, 4);
+        }
+    }
+    CU_CHECK(c, cudaMemcpy(c->d_blob, host.data(), total * sizeof(float), cudaMemcpyHostToDevice));
+    // transposed copies for the per-sample chain
+    const size_t D = c->D, H = c->H;
+    std::vector<float> wmuT(H * D), w2T(H * 2 * D);
+    const float* wmu = host.data() + off[10];
+    const float* w2 = host.data() + off[17];
+    for (size_t d = 0; d < D; ++d)
+        for (size_t i = 0; i < H; ++i) wmuT[i * D + d] = wmu[d * H + i];
+    for (size_t r = 0; r < 2 * D; ++r)
+        for (size_t i = 0; i < H; ++i) w2T[i * 2 * D + r] = w2[r * H + i];
+    CU_CHECK(c, cudaMemcpy(c->d_WmuT, wmuT.data(), wmuT.size() * sizeof(float), cudaMemcpyHostToDevice));
+    CU_CHECK(c, cudaMemcpy(c->d_W2T, w2T.data(), w2T.size() * sizeof(float), cudaMemcpyHostToDevice));
+
+    ModelDev& m = c->m;
+    m.N = c->N; m.D = c->D; m.H = c->H; m.W = c->W;
+    const float* b = c->d_blob;
+    m.Wxf = b + off[0]; m.Whf = b + off[1]; m.bf = b + off[2]; m.a0 = b + off[3];
+    m.Wxb = b + off[4]; m.Whb = b + off[5]; m.bb = b + off[6]; m.b0 = b + off[7];
+    m.Wz = b + off[8]; m.bz = b + off[9]; m.WmuT = c->d_WmuT; m.bmu = b + off[11];
+    m.Wsig = b + off[12]; m.bsig = b + off[13]; m.z0 = b + off[14];
+    m.W1 = b + off[15]; m.b1 = b + off[16]; m.W2T = c->d_W2T; m.b2 = b + off[18];
+    m.W3 = b + off[19]; m.b3 = b + off[20]; m.W4 = b + off[21]; m.b4 = b + off[22];
+    c->weights_loaded = true;
+    return CUTOFF_OK;
+}
+
+static int push_common(cutoff_ctx* c, const float* dev_src) {
+    k_push<<<1, kPushThreads, 0, c->stream>>>(dev_src, c->d_ring, c->d_state, c->N, c->W);
+    c->launches += 1;
+    CU_CHECK(c, cudaGetLastError());
+    c->pushes += 1;
+    return CUTOFF_OK;
+}
+
+int cutoff_push_async(cutoff_ctx* c, const float* runtimes_sec_device) {
+    if (!c || !runtimes_sec_device) return CUTOFF_ERR_BAD_ARG;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    return push_common(c, runtimes_sec_device);
+}
+
+int cutoff_push(cutoff_ctx* c, const float* runtimes_sec, int on_device, const uint8_t* censored) {
+    if (!c || !runtimes_sec) return CUTOFF_ERR_BAD_ARG;
+    if (censored) return CUTOFF_ERR_UNSUPPORTED;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (!on_device) {
+        for (int j = 0; j < c->N; ++j)
+            if (!(runtimes_sec[j] > 0.0f) || !std::isfinite(runtimes_sec[j])) return CUTOFF_ERR_BAD_VALUE;
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));       // the landing buffer may still be in use
+        std::memcpy(c->h_stage, runtimes_sec, sizeof(float) * c->N);
+        CU_CHECK(c, cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, cudaMemcpyHostToDevice, c->stream));
+        return push_common(c, c->d_stage);
+    }
+    const int rc = push_common(c, runtimes_sec);
+    if (rc) return rc;
+    CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    if (c->h_state->error_flags & kErrBadValue) {
+        // the kernel left the window untouched; clear the flag and undo the host-side count
+        c->pushes = c->h_state->push_count;
+        CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
+        return CUTOFF_ERR_BAD_VALUE;
+    }
+    return CUTOFF_OK;
+}
+
+int cutoff_predict_async(cutoff_ctx* c) {
+    if (!c) return CUTOFF_ERR_BAD_ARG;
+    if (!c->weights_loaded) return CUTOFF_ERR_STATE;
+    if (c->pending) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    c->pending = true;
+    c->pending_warmup = c->pushes < static_cast<uint32_t>(c->W);
+    if (c->pending_warmup) {
+        // nothing to compute; still read the state so that a bad device push is reported
+        CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+        return CUTOFF_OK;
+    }
+    const int rc = enqueue_decision(c);
+    if (rc) c->pending = false;
+    return rc;
+}
+
+int cutoff_fetch(cutoff_ctx* c, int32_t* c_out) {
+    if (!c || !c_out) return CUTOFF_ERR_BAD_ARG;
+    if (!c->pending) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    c->pending = false;
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    if (c->h_state->error_flags & kErrBadValue) {
+        c->pushes = c->h_state->push_count;
+        CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
+        return CUTOFF_ERR_BAD_VALUE;
+    }
+    if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
+    if (c->pending_warmup) {
+        *c_out = c->N;
+        return CUTOFF_WARMUP;
+    }
+    const int rc = collect_timing(c);
+    if (rc) return rc;
+    c->have_result = true;
+    *c_out = c->h_state->c_star;
+    return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
+}
+
+int cutoff_predict(cutoff_ctx* c, int32_t* c_out) {
+    if (!c || !c_out) return CUTOFF_ERR_BAD_ARG;
+    const int rc = cutoff_predict_async(c);
+    if (rc < 0) return rc;
+    return cutoff_fetch(c, c_out);
+}
+
+int cutoff_get_stats(cutoff_ctx* c, float* e_out, float* omega_out) {
+    if (!c) return CUTOFF_ERR_BAD_ARG;
+    if (!c->have_result) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (e_out) CU_CHECK(c, cudaMemcpyAsync(e_out, c->d_E, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
+    if (omega_out)
+        CU_CHECK(c, cudaMemcpyAsync(omega_out, c->d_omega, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    return CUTOFF_OK;
+}
+
+int cutoff_get_partial_sums(cutoff_ctx* c, double* sums) {
+    if (!c || !sums) return CUTOFF_ERR_BAD_ARG;
+    if (!c->have_result) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaMemcpyAsync(sums, c->d_sums, sizeof(double) * c->N, cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    return CUTOFF_OK;
+}
+
+int cutoff_decide_from_sums(cutoff_ctx* c, const double* sums, int32_t* c_out) {
+    if (!c || !sums || !c_out) return CUTOFF_ERR_BAD_ARG;
+    if (c->pending) return CUTOFF_ERR_STATE;
+    if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaMemcpyAsync(c->d_sums, sums, sizeof(double) * c->N, cudaMemcpyHostToDevice, c->stream));
+    const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
+    k_decide<<<1, kDecideThreads, 0, c->stream>>>(c->d_sums, c->N, 1.0 / static_cast<double>(total), c->d_state, 0,
+                                                  c->d_E, c->d_omega);
+    c->launches += 1;
+    CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    c->have_result = true;
+    *c_out = c->h_state->c_star;
+    return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
+}
+
+int cutoff_reset(cutoff_ctx* c) {
+    if (!c) return CUTOFF_ERR_BAD_ARG;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
+    CU_CHECK(c, cudaMemsetAsync(c->d_ring, 0, sizeof(float) * c->W * c->N, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    c->pushes = 0;
+    c->pending = false;
+    c->have_result = false;
+    return CUTOFF_OK;
+}
+
+int cutoff_save_state(cutoff_ctx* c, void* buf, size_t* nbytes) {
+    if (!c || !nbytes) return CUTOFF_ERR_BAD_ARG;
+    const size_t need = 4 * sizeof(uint32_t) + sizeof(DevState) + sizeof(float) * c->W * c->N;
+    if (!buf) { *nbytes = need; return CUTOFF_OK; }
+    if (*nbytes < need) return CUTOFF_ERR_BAD_ARG;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    char* p = static_cast<char*>(buf);
+    const uint32_t hdr[4] = {0x53465443u /* "CTFS" */, 1u, static_cast<uint32_t>(c->N), static_cast<uint32_t>(c->W)};
+    std::memcpy(p, hdr, sizeof(hdr));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    CU_CHECK(c, cudaMemcpy(p + sizeof(hdr), c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost));
+    CU_CHECK(c, cudaMemcpy(p + sizeof(hdr) + sizeof(DevState), c->d_ring, sizeof(float) * c->W * c->N,
+                           cudaMemcpyDeviceToHost));
+    *nbytes = need;
+    return CUTOFF_OK;
+}
+
+int cutoff_restore_state(cutoff_ctx* c, const void* buf, size_t nbytes) {
+    if (!c || !buf) return CUTOFF_ERR_BAD_ARG;
+    const size_t need = 4 * sizeof(uint32_t) + sizeof(DevState) + sizeof(float) * c->W * c->N;
+    if (nbytes != need) return CUTOFF_ERR_BAD_ARG;
+    const char* p = static_cast<const char*>(buf);
+    uint32_t hdr[4];
+    std::memcpy(hdr, p, sizeof(hdr));
+    if (hdr[0] != 0x53465443u || hdr[1] != 1u || hdr[2] != static_cast<uint32_t>(c->N) ||
+        hdr[3] != static_cast<uint32_t>(c->W))
+        return CUTOFF_ERR_BAD_ARG;
+    DevState s;
+    std::memcpy(&s, p + sizeof(hdr), sizeof(s));
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    CU_CHECK(c, cudaMemcpy(c->d_state, &s, sizeof(DevState), cudaMemcpyHostToDevice));
+    CU_CHECK(c, cudaMemcpy(c->d_ring, p + sizeof(hdr) + sizeof(DevState), sizeof(float) * c->W * c->N,
+                           cudaMemcpyHostToDevice));
+    c->pushes = s.push_count;
+    c->pending = false;
+    c->have_result = false;
+    return CUTOFF_OK;
+}
+
+int cutoff_set_timing(cutoff_ctx* c, int on) {
+    if (!c) return CUTOFF_ERR_BAD_ARG;
+    if (on && (c->cfg.flags & CUTOFF_FLAG_GRAPH)) return CUTOFF_ERR_UNSUPPORTED;
+    c->timing = on != 0;
+    return CUTOFF_OK;
+}
+
+int cutoff_get_timing(cutoff_ctx* c, float* ms, int cap) {
+    if (!c || !ms || cap < 0) return CUTOFF_ERR_BAD_ARG;
+    for (int i = 0; i < kNumStages && i < cap; ++i) ms[i] = c->stage_ms[i];
+    return kNumStages;
+}
+
+int64_t cutoff_launch_count(cutoff_ctx* c) { return c ? c->launches : 0; }
+
+int cutoff_set_option(cutoff_ctx* c, const char* name, int64_t value) {
+    if (!c || !name) return CUTOFF_ERR_BAD_ARG;
+    if (c->pending) return CUTOFF_ERR_STATE;
+    if (std::strcmp(name, "pass_rows") == 0) {
+        if (value < 1024) return CUTOFF_ERR_BAD_ARG;
+        plan_chunks(c, static_cast<int>(value));
+        return CUTOFF_OK;
+    }
+    return CUTOFF_ERR_BAD_ARG;
+}
+
+// ---- test hooks --------------------------------------------------------------------------------
+
+namespace {
+__global__ void k_debug_normals(uint32_t seed_lo, uint32_t seed_hi, uint32_t step, uint32_t stream, uint32_t k0,
+                                int64_t count, int nq, int n_elems, float* __restrict__ normals,
+                                uint32_t* __restrict__ words) {
+    const int64_t idx = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= count * nq) return;
+    const int64_t k = idx / nq;
+    const int q = static_cast<int>(idx % nq);
+    const Philox4 r = philox4x32_10(q, k0 + static_cast<uint32_t>(k), stream, step, seed_lo, seed_hi);
+    if (words) {
+        uint32_t* w = words + idx * 4;
+        w[0] = r.x; w[1] = r.y; w[2] = r.z; w[3] = r.w;
+    }
+    if (normals) {
+        float e[4];
+        box_muller(r.x, r.y, e[0], e[1]);
+        box_muller(r.z, r.w, e[2], e[3]);
+        for (int c = 0; c < 4; ++c)
+            if (4 * q + c < n_elems) normals[k * n_elems + 4 * q + c] = e[c];
+    }
+}
+}  // namespace
+
+int cutoff_debug_normals(int device, uint64_t seed, uint32_t step, uint32_t stream, int64_t k0, int64_t count,
+                         int32_t n_elems, float* normals_out, uint32_t* words_out) {
+    if (device < 0 || k0 < 0 || count < 1 || n_elems < 1 || k0 + count > (1ll << 32)) return CUTOFF_ERR_BAD_ARG;
+    if (!normals_out && !words_out) return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    CU_CHECK(none, cudaSetDevice(device));
+    const int nq = (n_elems + 3) / 4;
+    float* d_n = nullptr;
+    uint32_t* d_w = nullptr;
+    int rc = CUTOFF_OK;
+    if (normals_out && cudaMalloc(&d_n, sizeof(float) * count * n_elems) != cudaSuccess) rc = CUTOFF_ERR_NOMEM;
+    if (!rc && words_out && cudaMalloc(&d_w, sizeof(uint32_t) * count * nq * 4) != cudaSuccess) rc = CUTOFF_ERR_NOMEM;
+    if (!rc) {
+        const int64_t threads = count * nq;
+        k_debug_normals<<<static_cast<unsigned>(ceil_div64(threads, 256)), 256>>>(
+            static_cast<uint32_t>(seed), static_cast<uint32_t>(seed >> 32), step, stream, static_cast<uint32_t>(k0),
+            count, nq, n_elems, d_n, d_w);
+        if (cudaDeviceSynchronize() != cudaSuccess) rc = CUTOFF_ERR_CUDA;
+    }
+    if (!rc && normals_out &&
+        cudaMemcpy(normals_out, d_n, sizeof(float) * count * n_elems, cudaMemcpyDeviceToHost) != cudaSuccess)
+        rc = CUTOFF_ERR_CUDA;
+    if (!rc && words_out &&
+        cudaMemcpy(words_out, d_w, sizeof(uint32_t) * count * nq * 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+        rc = CUTOFF_ERR_CUDA;
+    cudaFree(d_n);
+    cudaFree(d_w);
+    return rc;
+}
+
+int cutoff_debug_samples(cutoff_ctx* c, int64_t k0, int64_t count, float* x_out) {
+    if (!c || !x_out || k0 < 0 || count < 1 || k0 + count > c->S) return CUTOFF_ERR_BAD_ARG;
+    if (!c->weights_loaded || c->pending) return CUTOFF_ERR_STATE;
+    if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    launch_encoder(c);
+    for (int64_t done = 0; done < count; done += c->chunk_rows) {
+        const int n = static_cast<int>(count - done < c->chunk_rows ? count - done : c->chunk_rows);
+        const uint32_t base = static_cast<uint32_t>(c->cfg.sample_offset + k0 + done);
+        launch_chain(c, base, n);
+        launch_emission(c, base, n);
+        CU_CHECK(c, cudaMemcpy2DAsync(x_out + done * c->N, sizeof(float) * c->N, c->d_x, sizeof(float) * c->ldx,
+                                      sizeof(float) * c->N, n, cudaMemcpyDeviceToHost, c->stream));
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    }
+    CU_CHECK(c, cudaGetLastError());
+    return CUTOFF_OK;
+}
+
+int cutoff_debug_sort(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t n, float* keys_out, int32_t* perm_out) {
+    if (!c || !rows || !keys_out || !perm_out || n_rows < 1 || n < 1 || n > 4096 || n_rows > (1 << 24))
+        return CUTOFF_ERR_BAD_ARG;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    const size_t elems = static_cast<size_t>(n_rows) * n;
+    float *d_rows = nullptr, *d_keys = nullptr;
+    int* d_perm = nullptr;
+    int rc = CUTOFF_OK;
+    if (cudaMalloc(&d_rows, elems * 4) != cudaSuccess || cudaMalloc(&d_keys, elems * 4) != cudaSuccess ||
+        cudaMalloc(&d_perm, elems * 4) != cudaSuccess)
+        rc = CUTOFF_ERR_NOMEM;
+    if (!rc && cudaMemcpyAsync(d_rows, rows, elems * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess)
+        rc = CUTOFF_ERR_CUDA;
+    if (!rc) {
+        const int P = next_pow2(n) < 32 ? 32 : next_pow2(n);
+        const int rows_i = static_cast<int>(n_rows);
+        const int grid_w = ceil_div(rows_i, kSortWarps) < 4 * c->sm_count ? ceil_div(rows_i, kSortWarps) : 4 * c->sm_count;
+        const int grid_c = rows_i < 4 * c->sm_count ? rows_i : 4 * c->sm_count;
+        switch (P) {
+            case 32: k_debug_sort_warp<1><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            case 64: k_debug_sort_warp<2><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            case 128: k_debug_sort_warp<4><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            case 256: k_debug_sort_warp<8><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            case 512: k_debug_sort_warp<16><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            case 1024: k_debug_sort_warp<32><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            default:
+                k_debug_sort_cta<<<grid_c, kSortCtaThreads, P * sizeof(unsigned long long), c->stream>>>(
+                    d_rows, n, P, rows_i, d_keys, d_perm);
+        }
+        c->launches += 1;
+        if (cudaMemcpyAsync(keys_out, d_keys, elems * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+            cudaMemcpyAsync(perm_out, d_perm, elems * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+            cudaStreamSynchronize(c->stream) != cudaSuccess)
+            rc = CUTOFF_ERR_CUDA;
+    }
+    if (rc == CUTOFF_ERR_CUDA) c->last_error = cudaGetErrorString(cudaGetLastError());
+    cudaFree(d_rows); cudaFree(d_keys); cudaFree(d_perm);
+    return rc;
+}
+
+}  // extern "C"

@@ -1,0 +1,284 @@
+"""Parity of the CUDA library with the CPU oracle, through the C ABI, on a real GPU.
+
+Tolerances (derived in the design doc):
+  noise words            bit-exact
+  standard normals       2e-6 * max(1, |eps|)
+  sampled run-times      rel 1e-5 (fp32 path) or 2e-3 (tf32 / bf16-weight tensor-core path),
+                         relative to max(|x|, mean |x|)
+  expected order stats   rel 1e-4, relative to max(|E_j|, |E_N|)
+  cutoff                 exact, unless the oracle's two best throughputs differ by less than 1e-4 relative
+  sort permutation       bit-exact
+"""
+import numpy as np
+import pytest
+
+from oracle import cutoff_oracle as O
+from paper_1803_04209_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+SEED = 0x5EEDC0FFEE123
+TOL_X = {0: 1e-5, 1: 2e-3, 2: 2e-3}
+TOL_E = 1e-4
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    import torch
+    assert torch.cuda.is_available(), "these tests need a GPU"
+    build.build()
+    return binding.load_library()
+
+
+def make_pair(name, S=None, steps=None, offsets=True, precision=None, seed=SEED, **kw):
+    wl = inputs.WORKLOADS[name]
+    S = S or wl.S
+    w = inputs.workload_weights(wl, offsets=offsets)
+    trace = inputs.workload_trace(wl, steps)
+    prec = wl.precision if precision is None else precision
+    gpu = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=prec, seed=seed, **kw)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, wl.lag, S, seed=seed)
+    for x in trace:
+        gpu.push(x)
+        orc.push(x)
+    return wl, gpu, orc, prec
+
+
+def assert_samples_close(x_gpu, x_orc, tol):
+    floor = np.abs(x_orc).mean()
+    err = np.abs(x_gpu.astype(np.float64) - x_orc) / np.maximum(np.abs(x_orc), floor)
+    assert np.all(np.isfinite(x_gpu))
+    assert err.max() <= tol, f"max relative error {err.max():.3e} > {tol:.1e}"
+
+
+def assert_decision_close(gpu, orc_result, N):
+    code_o, c_o, e_o, om_o = orc_result
+    code_g, c_g = gpu.predict()
+    e_g, om_g = gpu.get_stats()
+    assert code_g == code_o
+    denom = np.maximum(np.abs(e_o), np.abs(e_o[-1]))
+    assert np.max(np.abs(e_g - e_o) / denom) <= TOL_E
+    assert np.all(np.diff(e_g) >= 0)
+    finite = np.isfinite(om_o)
+    clearly_positive = e_o > TOL_E * np.abs(e_o[-1])
+    assert np.array_equal(np.isfinite(om_g)[clearly_positive | (e_o < -TOL_E * np.abs(e_o[-1]))],
+                          finite[clearly_positive | (e_o < -TOL_E * np.abs(e_o[-1]))])
+    both = finite & np.isfinite(om_g) & clearly_positive
+    assert np.max(np.abs(om_g[both] - om_o[both]) / np.abs(om_o[both])) <= 10 * TOL_E
+    if c_g != c_o:
+        # allowed only when the oracle's two best throughputs are within tolerance of each other
+        top = np.sort(om_o[finite])[-2:]
+        assert (top[1] - top[0]) <= TOL_E * abs(top[1]), f"cutoff {c_g} != oracle {c_o}"
+        assert abs(om_o[c_g - 1] - top[1]) <= TOL_E * abs(top[1])
+    return c_g
+
+
+# ----------------------------------------------------------------------------
+def test_noise_generator_bit_exact():
+    for (step, stream, k0, count, n) in ((0, 0, 0, 64, 16), (7, 0x200, 4_000_000_000, 33, 1024),
+                                          (123456, 0x100, 65500, 100, 7), (1, 3, 5, 1, 1)):
+        normals, words = binding.debug_normals(SEED, step, stream, k0, count, n)
+        k = np.arange(k0, k0 + count, dtype=np.uint64)
+        nq = (n + 3) // 4
+        ref_words = np.stack(O.philox4x32_10(np.arange(nq, dtype=np.uint64)[None, :], k[:, None], stream, step,
+                                             SEED & 0xFFFFFFFF, SEED >> 32), axis=-1)
+        assert np.array_equal(words.astype(np.uint64), ref_words)
+        ref = O.normals(SEED, step, stream, k, n)
+        assert np.max(np.abs(normals - ref) / np.maximum(1.0, np.abs(ref))) <= 2e-6
+
+
+def test_noise_generator_known_answer_on_gpu():
+    # counter (0, 0, 0, 0), key (0, 0): first published known-answer vector
+    _, words = binding.debug_normals(0, 0, 0, 0, 1, 4)
+    assert [int(v) for v in words[0, 0]] == [0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8]
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 16, 33, 158, 512, 1024, 1025, 2175, 4096])
+def test_sort_permutation_bit_exact(n):
+    rng = np.random.default_rng(n)
+    rows = [rng.integers(0, 50, size=n), rng.integers(-1000, 1000, size=n), np.full(n, 7),
+            np.arange(n)[::-1], np.arange(n), rng.integers(0, 3, size=n)]
+    rows += [rng.integers(-5, 5, size=n) for _ in range(11)]
+    rows = np.stack(rows).astype(np.float32) * np.float32(0.25)
+    rows[rows == 0] = 0.0          # no negative zeros
+    gpu = binding.Cutoff(16, 4, 32, 1, 64)
+    keys, perm = gpu.debug_sort(rows)
+    want_perm = np.argsort(rows, axis=1, kind="stable")
+    assert np.array_equal(perm, want_perm)
+    assert np.array_equal(keys, np.take_along_axis(rows, want_perm, axis=1))
+
+
+@pytest.mark.parametrize("name,S,offsets", [("tiny", 1024, True), ("tiny", 1024, False), ("n128", 2048, True),
+                                            ("n128", 777, False), ("n158", 512, True)])
+def test_sampled_runtimes_fp32(name, S, offsets):
+    wl, gpu, orc, prec = make_pair(name, S=S, offsets=offsets)
+    x_gpu = gpu.debug_samples(0, S)
+    x_orc = orc.samples(np.arange(S))
+    assert_samples_close(x_gpu, x_orc, TOL_X[prec])
+    # a window of samples from the middle gives the same rows (draws are addressed by sample index)
+    assert np.array_equal(gpu.debug_samples(100, 50), x_gpu[100:150])
+
+
+@pytest.mark.parametrize("name,S,offsets", [("tiny", 1024, True), ("tiny", 1024, False), ("n128", 4096, True),
+                                            ("n128", 1500, False), ("n158", 1024, True)])
+def test_decision_fp32(name, S, offsets):
+    wl, gpu, orc, prec = make_pair(name, S=S, offsets=offsets)
+    assert_decision_close(gpu, orc.predict(), wl.N)
+
+
+def test_wide_models_fp32_arithmetic():
+    # the large shapes with every product in fp32: isolates the non-tensor-core kernels
+    for name, S in (("n1024", 1536), ("n2175", 300), ("n4096", 300)):
+        wl, gpu, orc, prec = make_pair(name, S=S, steps=12, precision=0)
+        assert_samples_close(gpu.debug_samples(0, min(S, 256)), orc.samples(np.arange(min(S, 256))), 2e-5)
+        assert_decision_close(gpu, orc.predict(), wl.N)
+
+
+def test_streaming_loop_matches_oracle():
+    wl = inputs.WORKLOADS["tiny"]
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, 14)
+    gpu = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 512, seed=SEED)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, wl.lag, 512, seed=SEED)
+    for t, x in enumerate(trace):
+        code_o, c_o, e_o, _ = orc.predict()
+        code_g, c_g = gpu.predict()
+        assert code_g == code_o
+        if code_o == O.WARMUP:
+            assert c_g == wl.N == c_o
+        else:
+            e_g, _ = gpu.get_stats()
+            assert np.max(np.abs(e_g - e_o) / e_o[-1]) <= TOL_E
+            assert c_g == c_o
+        gpu.push(x)
+        orc.push(x)
+
+
+def test_device_pushes_equal_host_pushes():
+    import torch
+    wl = inputs.WORKLOADS["n128"]
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, 9)
+    a = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 256, seed=3)
+    b = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 256, seed=3)
+    a.load_weights(w)
+    b.load_weights(w)
+    dev = torch.from_numpy(trace).cuda()
+    torch.cuda.synchronize()
+    for t in range(trace.shape[0]):
+        a.push(trace[t])
+        if t % 2:
+            b.push(dev[t])
+        else:
+            b.push_async(dev[t])
+    assert a.predict() == b.predict()
+    assert np.array_equal(a.get_stats()[0], b.get_stats()[0])
+
+
+def test_pass_size_does_not_change_the_result():
+    wl, gpu, orc, _ = make_pair("n128", S=5000, steps=8)
+    ref = gpu.predict()
+    e_ref, _ = gpu.get_stats()
+    wl, gpu2, _, _ = make_pair("n128", S=5000, steps=8)
+    gpu2.set_option("pass_rows", 1024)
+    assert gpu2.predict() == ref
+    e2, _ = gpu2.get_stats()
+    assert np.max(np.abs(e2 - e_ref) / e_ref[-1]) <= 1e-6
+
+
+def test_sample_sharding_adds_up():
+    # two contexts that each draw half of the samples of one decision
+    wl = inputs.WORKLOADS["n128"]
+    S = 2048
+    _, whole, orc, _ = make_pair("n128", S=S, steps=8)
+    _, lo, _, _ = make_pair("n128", S=S // 2, steps=8, sample_offset=0, total_samples=S)
+    _, hi, _, _ = make_pair("n128", S=S // 2, steps=8, sample_offset=S // 2, total_samples=S)
+    assert np.array_equal(hi.debug_samples(0, 8), whole.debug_samples(S // 2, 8))   # global sample index
+    code, c = whole.predict()
+    lo.predict()
+    hi.predict()
+    total = lo.get_partial_sums() + hi.get_partial_sums()
+    assert np.allclose(total, whole.get_partial_sums(), rtol=1e-6)
+    code2, c2 = lo.decide_from_sums(total)
+    assert (code2, c2) == (code, c)
+    assert np.max(np.abs(lo.get_stats()[0] - whole.get_stats()[0]) / whole.get_stats()[0][-1]) <= 1e-6
+
+
+def test_state_save_restore_and_reset():
+    wl, gpu, orc, _ = make_pair("tiny", S=256, steps=7)
+    blob = gpu.save_state()
+    first = gpu.predict()
+    e_first, _ = gpu.get_stats()
+    gpu.push(inputs.workload_trace(wl, 8)[7])
+    gpu.restore_state(blob)
+    assert gpu.predict() == first
+    assert np.array_equal(gpu.get_stats()[0], e_first)
+    gpu.reset()
+    assert gpu.predict() == (binding.WARMUP, wl.N)
+
+
+def test_errors_are_codes_not_crashes():
+    wl = inputs.WORKLOADS["tiny"]
+    w = inputs.workload_weights(wl)
+    gpu = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 128)
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.predict()                                   # no weights yet
+    assert e.value.code == binding.ERR_STATE
+    blob = binding.pack_weights(w, wl.N, wl.D, wl.H)
+    for bad in (blob[:-4], b"\0" * len(blob), blob[:8] + b"\x11\0\0\0" + blob[12:]):
+        with pytest.raises(binding.CutoffError) as e:
+            gpu.load_weights(bad)
+        assert e.value.code == binding.ERR_BAD_BLOB
+    nan_blob = bytearray(blob)
+    nan_blob[24:28] = np.float32(np.nan).tobytes()
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.load_weights(bytes(nan_blob))
+    assert e.value.code == binding.ERR_BAD_BLOB
+    gpu.load_weights(w)
+    assert gpu.predict() == (binding.WARMUP, wl.N)
+    good = np.ones(wl.N, dtype=np.float32)
+    for bad_value in (0.0, -1.0, np.nan, np.inf):
+        x = good.copy()
+        x[5] = bad_value
+        with pytest.raises(binding.CutoffError) as e:
+            gpu.push(x)
+        assert e.value.code == binding.ERR_BAD_VALUE
+        import torch
+        with pytest.raises(binding.CutoffError) as e:
+            gpu.push(torch.from_numpy(x).cuda())
+        assert e.value.code == binding.ERR_BAD_VALUE
+    # rejected pushes leave no trace: two good pushes complete the window
+    gpu.push(good)
+    assert gpu.predict() == (binding.WARMUP, wl.N)
+    gpu.push(good)
+    assert gpu.predict()[0] == binding.OK
+    import ctypes as C
+    flag = (C.c_uint8 * wl.N)()
+    assert gpu._lib.cutoff_push(gpu._h, good.ctypes.data, 0, flag) == binding.ERR_UNSUPPORTED
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.fetch()                                     # nothing enqueued
+    assert e.value.code == binding.ERR_STATE
+
+
+def test_degenerate_and_equal_times():
+    # every expected time negative -> c = N with the informational code; equal deterministic times -> c = N
+    wl = inputs.WORKLOADS["tiny"]
+    w = inputs.workload_weights(wl)
+    w["W4"][:] = 0.0
+    w["b4"][: wl.N] = -1.0
+    gpu = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 128)
+    gpu.load_weights(w)
+    for x in inputs.workload_trace(wl, 3):
+        gpu.push(x)
+    assert gpu.predict() == (binding.DEGENERATE, wl.N)
+    e, om = gpu.get_stats()
+    assert np.all(e < 0) and np.all(np.isneginf(om))
+    w["b4"][: wl.N] = 0.75
+    w["b4"][wl.N:] = -150.0
+    gpu.load_weights(w)
+    assert gpu.predict() == (binding.OK, wl.N)
+    e, om = gpu.get_stats()
+    s = 2.0 * inputs.workload_trace(wl, 3)[:2].astype(np.float64).mean()
+    assert np.allclose(e, 0.75 * s, rtol=1e-6)
