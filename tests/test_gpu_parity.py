@@ -130,7 +130,7 @@ def test_decision_fp32(name, S, offsets):
 def test_wide_models_fp32_arithmetic():
     # the large shapes with every product in fp32: isolates the non-tensor-core kernels
     for name, S in (("n1024", 1536), ("n2175", 300), ("n4096", 300)):
-        wl, gpu, orc, prec = make_pair(name, S=S, steps=12, precision=0)
+        wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 7, precision=0)
         assert_samples_close(gpu.debug_samples(0, min(S, 256)), orc.samples(np.arange(min(S, 256))), 2e-5)
         assert_decision_close(gpu, orc.predict(), wl.N)
 
