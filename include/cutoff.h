@@ -60,7 +60,8 @@ enum {
     CUTOFF_ERR_UNSUPPORTED = -5,
     CUTOFF_ERR_NOMEM = -6,
     CUTOFF_ERR_STATE = -7,      /* call order: weights not loaded, nothing predicted yet, ...      */
-    CUTOFF_ERR_TIMEOUT = -8     /* a bounded device-side wait gave up (tensor-core pipeline)        */
+    CUTOFF_ERR_TIMEOUT = -8,    /* a bounded device-side wait gave up (tensor-core pipeline)        */
+    CUTOFF_ERR_TOO_LARGE = -9   /* the request exceeds a fixed built-in capacity                    */
 };
 
 enum {
@@ -190,6 +191,38 @@ int cutoff_debug_normals(int device, uint64_t seed, uint32_t step, uint32_t stre
 int cutoff_debug_samples(cutoff_ctx* ctx, int64_t k0, int64_t count, float* x_out);
 int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n,
                       float* keys_out, int32_t* perm_out);
+
+/* ---- allocation-free entry point ---------------------------------------------------------------
+ * The paper has no counterpart for this call.  It serves programs that may not allocate device
+ * memory at the time they need order statistics: a server that handed all of the GPU's memory to
+ * its own pool at start-up (a late cudaMalloc there fails or fragments the pool), a control loop
+ * that cannot afford the device-wide synchronisation an allocation may imply, or code under a
+ * "nothing is allocated after initialisation" rule.  Such a caller already holds its predictive
+ * samples and only wants them sorted and summed.
+ *
+ * cutoff_sorted_row_sums_static sorts the first n entries of each of n_rows rows ascending and adds
+ * the sorted rows position by position:   sums[j] = sum over rows of (j-th smallest entry of the row).
+ * Dividing by n_rows gives the Monte-Carlo expected order statistics of Section 3.1.1.
+ *   device    CUDA device ordinal (0..63) that owns x, sums and stream
+ *   x         device, n_rows x ldx floats, row-major; entries beyond n in a row are ignored
+ *   n_rows    1 .. 2^31-1;   n  1 .. CUTOFF_STATIC_MAX_N;   ldx >= n
+ *   sums      device, n doubles, overwritten
+ *   stream    cudaStream_t to run on (NULL = default stream); the call only enqueues work
+ * The call performs no cudaMalloc, cudaFree or other allocating routine.  Its only scratch is a
+ * fixed array of CUTOFF_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that
+ * loads the library holds that much memory until the process exits.  n above the limit returns
+ * CUTOFF_ERR_TOO_LARGE and does nothing.
+ * The first call on a device looks up the array's device address (a one-time set-up step that
+ * loads the library's code on that device); make that first call before starting any stream
+ * capture.  All calls on a device share the one array, and it keeps what the last call left in
+ * it: each call overwrites every scratch row it later reads, so nothing needs clearing, but two
+ * calls whose work overlaps on the GPU (different streams, or different host threads) race on it.
+ * Issue them on one stream, or order them with events.  Not thread-safe with respect to its
+ * first call on a device.  Errors: BAD_ARG, TOO_LARGE, CUDA. */
+#define CUTOFF_STATIC_MAX_N 1024
+#define CUTOFF_STATIC_SCRATCH_BYTES (256 * 1024 * 4)
+int cutoff_sorted_row_sums_static(int device, const float* x, int64_t n_rows, int32_t n, int32_t ldx,
+                                  double* sums, void* stream);
 
 #ifdef __cplusplus
 }

@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(PKG_DIR, "libcutoff.so")
 
 OK, WARMUP, DEGENERATE = 0, 1, 2
 ERR_BAD_ARG, ERR_BAD_BLOB, ERR_BAD_VALUE, ERR_CUDA = -1, -2, -3, -4
-ERR_UNSUPPORTED, ERR_NOMEM, ERR_STATE, ERR_TIMEOUT = -5, -6, -7, -8
+ERR_UNSUPPORTED, ERR_NOMEM, ERR_STATE, ERR_TIMEOUT, ERR_TOO_LARGE = -5, -6, -7, -8, -9
+STATIC_MAX_N = 1024
 PRECISION_FP32, PRECISION_TF32, PRECISION_BF16W = 0, 1, 2
 FLAG_GRAPH = 1
 BLOB_MAGIC = 0x31465443
@@ -29,7 +30,7 @@ EXPORTS = (
     "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
-    "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_sort",
+    "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_sort", "cutoff_sorted_row_sums_static",
 )
 
 
@@ -87,6 +88,7 @@ def load_library(path: str | None = None) -> C.CDLL:
                                            C.c_int32, vp, vp]),
         "cutoff_debug_samples": (C.c_int, [vp, C.c_int64, C.c_int64, vp]),
         "cutoff_debug_sort": (C.c_int, [vp, vp, C.c_int64, C.c_int32, vp, vp]),
+        "cutoff_sorted_row_sums_static": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)          # AttributeError if the library does not export it
@@ -257,3 +259,18 @@ def debug_normals(seed: int, step: int, stream: int, k0: int, count: int, n_elem
     if rc < 0:
         raise CutoffError(rc, "cutoff_debug_normals")
     return normals, words
+
+
+def sorted_row_sums_static(x, sums, n: int | None = None, stream: int | None = None) -> int:
+    """Allocation-free sum of sorted rows: x (torch CUDA fp32 [rows, ldx]) -> sums (torch CUDA fp64 [n]).
+
+    Both tensors belong to the caller; the call itself allocates nothing (its scratch is a fixed
+    array inside the library).  Returns the library's code; raises on an error code.
+    """
+    lib = load_library()
+    n = x.shape[1] if n is None else n
+    rc = lib.cutoff_sorted_row_sums_static(x.device.index or 0, x.data_ptr(), x.shape[0], n, x.stride(0),
+                                           sums.data_ptr(), stream or None)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_sorted_row_sums_static")
+    return rc

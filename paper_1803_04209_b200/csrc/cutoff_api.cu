@@ -269,6 +269,7 @@ const char* cutoff_strerror(int code) {
         case CUTOFF_ERR_NOMEM: return "out of device memory";
         case CUTOFF_ERR_STATE: return "call out of order";
         case CUTOFF_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case CUTOFF_ERR_TOO_LARGE: return "request exceeds a fixed built-in capacity (see CUTOFF_STATIC_MAX_N)";
         default: return "unknown code";
     }
 }
@@ -732,3 +733,56 @@ int cutoff_debug_sort(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t 
 }
 
 }  // extern "C"
+
+// ---- allocation-free entry point -------------------------------------------------------------
+
+namespace {
+constexpr int kStaticParts = 256;     // partial rows (= most CTAs the sort kernel may use here)
+static_assert(kStaticParts * CUTOFF_STATIC_MAX_N * sizeof(float) == CUTOFF_STATIC_SCRATCH_BYTES, "scratch size");
+
+// Scratch of cutoff_sorted_row_sums_static: one partial sum row per CTA.  Lives in the library
+// image, one copy per GPU.  In host code this name is only a handle for cudaGetSymbolAddress;
+// the kernels get the device address found at set-up.
+static __device__ __align__(256) float g_static_partial[kStaticParts * CUTOFF_STATIC_MAX_N];
+
+constexpr int kMaxDevices = 64;
+float* g_static_partial_addr[kMaxDevices] = {};   // device address per GPU, filled on first use
+
+template <int E>
+void launch_static_sort(const float* x, int ldx, int n, int n_rows, int grid, float* partial, cudaStream_t stream) {
+    k_sort_sum_warp<E><<<grid, kSortWarps * 32, 0, stream>>>(x, ldx, n, n_rows, partial);
+}
+}  // namespace
+
+extern "C" int cutoff_sorted_row_sums_static(int device, const float* x, int64_t n_rows, int32_t n, int32_t ldx,
+                                             double* sums, void* stream) {
+    if (device < 0 || device >= kMaxDevices || !x || !sums || n_rows < 1 || n_rows > 0x7fffffffll || n < 1 || ldx < n)
+        return CUTOFF_ERR_BAD_ARG;
+    if (n > CUTOFF_STATIC_MAX_N) return CUTOFF_ERR_TOO_LARGE;
+    if (cudaSetDevice(device) != cudaSuccess) return CUTOFF_ERR_CUDA;
+    if (!g_static_partial_addr[device]) {
+        // once per device, with that device current: translate the symbol into a device address
+        float* addr = nullptr;
+        if (cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_static_partial) != cudaSuccess || !addr)
+            return CUTOFF_ERR_CUDA;
+        g_static_partial_addr[device] = addr;
+    }
+    float* partial = g_static_partial_addr[device];
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int rows = static_cast<int>(n_rows);
+    const int want = ceil_div(rows, kSortWarps);
+    const int grid = want < kStaticParts ? want : kStaticParts;
+    const int P = next_pow2(n) < 32 ? 32 : next_pow2(n);
+    // every CTA of the grid writes its whole partial row (zeros if it had no sample), and the
+    // column sum reads exactly `grid` rows: stale contents of the shared array are never read
+    switch (P) {
+        case 32: launch_static_sort<1>(x, ldx, n, rows, grid, partial, s); break;
+        case 64: launch_static_sort<2>(x, ldx, n, rows, grid, partial, s); break;
+        case 128: launch_static_sort<4>(x, ldx, n, rows, grid, partial, s); break;
+        case 256: launch_static_sort<8>(x, ldx, n, rows, grid, partial, s); break;
+        case 512: launch_static_sort<16>(x, ldx, n, rows, grid, partial, s); break;
+        default: launch_static_sort<32>(x, ldx, n, rows, grid, partial, s); break;
+    }
+    k_colsum<<<ceil_div(n, 256), 256, 0, s>>>(partial, grid, n, sums);
+    return cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
+}
