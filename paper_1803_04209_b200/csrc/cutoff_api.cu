@@ -11,6 +11,7 @@
 #include "common.cuh"
 #include "kernels_model.cuh"
 #include "kernels_sort.cuh"
+#include "emit_tc.cuh"
 
 using namespace cutoff;
 
@@ -53,6 +54,10 @@ struct cutoff_ctx {
     double* d_sums = nullptr;       // [N]
     float* d_E = nullptr;           // [N]
     float* d_omega = nullptr;       // [N]
+
+    CUtensorMap map_v{};            // TMA view of d_v   [alloc_rows][H]
+    CUtensorMap map_w4{};           // TMA view of W4    [2N][H]
+    bool use_tc = false;            // emission output layer on tensor cores
 
     float* h_stage = nullptr;       // pinned [N]
     DevState* h_state = nullptr;    // pinned
@@ -176,7 +181,55 @@ void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
     c->launches += 1;
 }
 
+// 2-D fp32 tensor map over a row-major [rows][cols] matrix, boxes of 128 rows x 32 columns
+// (one 128-byte-swizzled K-major operand tile).  The driver entry point is looked up at run time.
+int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t rows, uint64_t cols) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        CU_CHECK(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (!fn || q != cudaDriverEntryPointSuccess) {
+            c->last_error = "cuTensorMapEncodeTiled is not available from this driver";
+            return CUTOFF_ERR_CUDA;
+        }
+        encode = reinterpret_cast<EncodeFn>(fn);
+    }
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * sizeof(float)};
+    const cuuint32_t box[2] = {tc::kBK, tc::kBM};
+    const cuuint32_t elem[2] = {1, 1};
+    const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box,
+                              elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        c->last_error = "cuTensorMapEncodeTiled failed with code " + std::to_string(static_cast<int>(r));
+        return CUTOFF_ERR_CUDA;
+    }
+    return CUTOFF_OK;
+}
+
+void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(tc::k_emit_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
+        attr_set = true;
+    }
+    tc::EmitArgs a;
+    a.b4 = c->m.b4; a.x = c->d_x; a.st = c->d_state;
+    a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    a.sample_base = sample_base; a.count = count; a.N = c->N; a.H = c->H; a.ldx = c->ldx;
+    const int tiles = ceil_div(c->N, tc::kBW) * ceil_div(count, tc::kBM);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    tc::k_emit_tc<<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(c->map_v, c->map_w4, a);
+    c->launches += 1;
+}
+
 void launch_emission(cutoff_ctx* c, uint32_t sample_base, int count) {
+    if (c->use_tc) { launch_emission_tc(c, sample_base, count); return; }
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     dim3 grid(ceil_div(c->N, kEmitTN), ceil_div(count, kEmitTM));
     k_emit_fma<<<grid, kEmitThreads, 0, c->stream>>>(c->m, c->d_v, c->d_state, key, sample_base, count, c->d_x, c->ldx);
@@ -310,17 +363,14 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     c->sm_count = prop.multiProcessorCount;
     if (chain_smem_floats(c->D, c->H, c->W) * sizeof(float) > 220 * 1024) return fail(CUTOFF_ERR_UNSUPPORTED);
 
-    // Default pass size: keep one pass's sample matrix within ~48 MB so it stays in L2.
-    int rows = static_cast<int>((48ll << 20) / (static_cast<int64_t>(c->ldx) * sizeof(float)));
-    rows = rows / 1024 * 1024;
-    if (rows < 1024) rows = 1024;
+    // Pass buffers hold up to 2 GiB of samples; by default one pass covers all S samples.
     {
-        // pass buffers are allocated for up to 2 GiB of samples so that larger passes can be tried
         int64_t cap = (2ll << 30) / (static_cast<int64_t>(c->ldx + c->H) * sizeof(float));
-        if (cap < rows) cap = rows;
+        if (cap < 1024) cap = 1024;
         c->alloc_rows = cap < c->S ? static_cast<int>(cap) : c->S;
     }
-    plan_chunks(c, rows);
+    plan_chunks(c, c->alloc_rows);
+    c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
 
     size_t blob_floats = 0;
     for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
@@ -340,6 +390,10 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_sums, sizeof(double) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_E, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_omega, sizeof(float) * c->N));
+    if (c->use_tc) {
+        const int rc = make_tile_map(c, &c->map_v, c->d_v, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
+        if (rc) return fail(rc);
+    }
     CREATE_CHECK(cudaMallocHost(&c->h_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMallocHost(&c->h_state, sizeof(DevState)));
     CREATE_CHECK(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
@@ -381,13 +435,15 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     std::vector<size_t> off(specs.size());
     size_t o = 0;
     for (size_t i = 0; i < specs.size(); ++i) { off[i] = o; o += specs[i].rows * specs[i].cols; }
-    if (c->cfg.precision == CUTOFF_PRECISION_BF16W) {
-        // round the output-layer weights to bf16 (nearest even), kept as fp32 bit patterns
+    if (c->use_tc) {
+        // Output-layer weights as the tensor cores will see them, kept as fp32 bit patterns:
+        // bf16 (nearest even) for the bf16-weight precision, else tf32 (nearest, ties away from zero).
         float* w4 = host.data() + off[21];
         for (size_t i = 0; i < specs[21].rows * specs[21].cols; ++i) {
             uint32_t u;
             std::memcpy(&u, &w4[i], 4);
-            u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
+            if (c->cfg.precision == CUTOFF_PRECISION_BF16W) u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
+            else u = (u + 0x1000u) & 0xFFFFE000u;
             std::memcpy(&w4[i], &u, 4);
         }
     }
@@ -413,6 +469,10 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     m.Wsig = b + off[12]; m.bsig = b + off[13]; m.z0 = b + off[14];
     m.W1 = b + off[15]; m.b1 = b + off[16]; m.W2T = c->d_W2T; m.b2 = b + off[18];
     m.W3 = b + off[19]; m.b3 = b + off[20]; m.W4 = b + off[21]; m.b4 = b + off[22];
+    if (c->use_tc) {
+        const int rc = make_tile_map(c, &c->map_w4, m.W4, 2ull * c->N, static_cast<uint64_t>(c->H));
+        if (rc) return rc;
+    }
     c->weights_loaded = true;
     return CUTOFF_OK;
 }

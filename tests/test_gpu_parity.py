@@ -135,6 +135,24 @@ def test_wide_models_fp32_arithmetic():
         assert_decision_close(gpu, orc.predict(), wl.N)
 
 
+@pytest.mark.parametrize("name,S", [("n1024", 1024), ("n1024", 130), ("n2175", 300), ("n4096", 384), ("stream", 256)])
+def test_sampled_runtimes_tensor_cores(name, S):
+    # output layer on tcgen05: operands rounded to tf32 (n4096: weights already bf16-representable)
+    wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 7)
+    assert prec in (1, 2)
+    x_gpu = gpu.debug_samples(0, S)
+    x_orc = orc.samples(np.arange(S))
+    assert_samples_close(x_gpu, x_orc, TOL_X[prec])
+    assert np.array_equal(gpu.debug_samples(S // 2, 7), x_gpu[S // 2: S // 2 + 7])
+
+
+@pytest.mark.parametrize("name,S,offsets", [("n1024", 4096, True), ("n1024", 1000, False), ("n2175", 512, True),
+                                            ("n4096", 1024, True)])
+def test_decision_tensor_cores(name, S, offsets):
+    wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 7, offsets=offsets)
+    assert_decision_close(gpu, orc.predict(), wl.N)
+
+
 def test_streaming_loop_matches_oracle():
     wl = inputs.WORKLOADS["tiny"]
     w = inputs.workload_weights(wl)
