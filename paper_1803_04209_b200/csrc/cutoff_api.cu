@@ -136,7 +136,13 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
 
 template <int E>
 void launch_sort_warp(cutoff_ctx* c, int count, float* partial) {
-    k_sort_sum_warp<E><<<c->sort_grid, kSortWarps * 32, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
+    static bool attr_set = false;
+    const size_t smem = sort_tma_smem_bytes<E>(c->ldx);
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_sort_sum_tma<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        attr_set = true;
+    }
+    k_sort_sum_tma<E><<<c->sort_grid, kSortWarps * 32, smem, c->stream>>>(c->d_x, c->ldx, c->N, count, partial, c->d_state);
 }
 
 int launch_sort(cutoff_ctx* c, int count, float* partial) {

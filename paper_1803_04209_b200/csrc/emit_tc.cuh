@@ -17,11 +17,14 @@
 #pragma once
 #include <cuda.h>
 
+#include "async.cuh"
 #include "common.cuh"
 #include "rng.cuh"
 
 namespace cutoff {
 namespace tc {
+
+using namespace cutoff::async;
 
 constexpr int kBM = 128;                 // samples per tile (TMEM lanes)
 constexpr int kBW = 128;                 // workers per tile
@@ -35,53 +38,9 @@ constexpr int kThreads = (2 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 2 * kBW;                // 256 columns per accumulator
 constexpr size_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 // instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128
 constexpr uint32_t kInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false if it gave up or if another role already aborted.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, DevState* st) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                atomicOr(&st->error_flags, kErrTimeout);
-                return false;
-            }
-        }
-    }
-}
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
@@ -290,15 +249,15 @@ __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__
                         const int j = jw + 4 * i;
                         if (j >= a.N) continue;
                         float eps[4];
-                        normal4(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
-                                a.key.seed_hi, eps);
+                        normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
+                                     a.key.seed_hi, eps);
                         float out[4];
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             const int jj = min(j + c, a.N - 1);
                             const float mean = __uint_as_float(mean_bits[4 * i + c]) + __ldg(a.b4 + jj);
                             const float logvar = __uint_as_float(logvar_bits[4 * i + c]) + __ldg(a.b4 + a.N + jj);
-                            out[c] = fmaf(expf(0.5f * logvar), eps[c], mean);
+                            out[c] = fmaf(exp_half_fast(logvar), eps[c], mean);
                         }
                         if (j + 3 < a.N) {
                             *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(out[0], out[1], out[2], out[3]);

@@ -3,61 +3,112 @@
 #pragma once
 #include <cfloat>
 #include <cmath>
+#include "async.cuh"
 #include "common.cuh"
 
 namespace cutoff {
 
 // Key types of the sorting network: float for the decision path; a 64-bit composite
 // (order-preserving key bits, original position) for the permutation test hook.
+// Besides min and max each type has an order-reversing involution ("reverse": negation for
+// floats, bitwise complement for unsigned integers).  A lane that has to keep the LARGER key of
+// an exchange holds its keys reversed, so that every lane executes the same min(own, reverse(other)).
 template <typename T> struct KeyOps;
 template <> struct KeyOps<float> {
+    using Flip = float;                                   // +1: as is, -1: reversed
     static __device__ __forceinline__ float lo(float a, float b) { return fminf(a, b); }
     static __device__ __forceinline__ float hi(float a, float b) { return fmaxf(a, b); }
     static __device__ __forceinline__ float pad() { return INFINITY; }
     static __device__ __forceinline__ float shfl_xor(float v, int mask) { return __shfl_xor_sync(0xffffffffu, v, mask); }
+    static __device__ __forceinline__ Flip identity() { return 1.0f; }
+    static __device__ __forceinline__ Flip flip_if(bool reversed) { return reversed ? -1.0f : 1.0f; }
+    static __device__ __forceinline__ Flip combine(Flip a, Flip b) { return a * b; }
+    static __device__ __forceinline__ float apply(float v, Flip f) { return v * f; }
+    static __device__ __forceinline__ float reverse(float v) { return -v; }
 };
 template <> struct KeyOps<unsigned long long> {
     using T = unsigned long long;
+    using Flip = unsigned long long;                      // 0: as is, ~0: reversed
     static __device__ __forceinline__ T lo(T a, T b) { return a < b ? a : b; }
     static __device__ __forceinline__ T hi(T a, T b) { return a < b ? b : a; }
     static __device__ __forceinline__ T pad() { return ~0ull; }
     static __device__ __forceinline__ T shfl_xor(T v, int mask) { return __shfl_xor_sync(0xffffffffu, v, mask); }
+    static __device__ __forceinline__ Flip identity() { return 0ull; }
+    static __device__ __forceinline__ Flip flip_if(bool reversed) { return reversed ? ~0ull : 0ull; }
+    static __device__ __forceinline__ Flip combine(Flip a, Flip b) { return a ^ b; }
+    static __device__ __forceinline__ T apply(T v, Flip f) { return v ^ f; }
+    static __device__ __forceinline__ T reverse(T v) { return ~v; }
 };
 
 // Bitonic sorting network over 32*E keys held by one warp, E keys per lane, key index
-// idx = lane*E + r ("blocked").  Exchange distances below E stay inside a lane's registers;
-// distances of E and more are lane exchanges by shuffle.  Ascending on exit.
+// idx = lane*E + r ("blocked").  Every merge of width k starts with the mirror exchange
+// idx <-> idx ^ (k-1) and continues with half-cleaners idx <-> idx ^ j, j = k/4 .. 1; the lower
+// index always keeps the smaller key, so no exchange depends on a direction flag.  Distances
+// below E stay inside a lane's registers (one min and one max per pair); distances of E and more
+// are lane exchanges by shuffle in the reversed-key form described above (one min per key; the
+// reversals are multiplications by +-1, which run on the otherwise idle FMA pipe).
+// Ascending on exit.
 template <typename T, int E>
 __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
     using Ops = KeyOps<T>;
+    typename Ops::Flip cur = Ops::identity();             // form the lane's keys are held in
 #pragma unroll
     for (int k = 2; k <= 32 * E; k <<= 1) {
+        if (k <= E) {
 #pragma unroll
-        for (int j = k >> 1; j > 0; j >>= 1) {
+            for (int r = 0; r < E; ++r) {
+                const int p = r ^ (k - 1);
+                if (p > r) {
+                    const T a = v[r], b = v[p];
+                    v[r] = Ops::lo(a, b);
+                    v[p] = Ops::hi(a, b);
+                }
+            }
+        } else {
+            const int lane_mask = k / E - 1;
+            const typename Ops::Flip want = Ops::flip_if((lane & (k / (2 * E))) != 0);
+            const typename Ops::Flip f = Ops::combine(want, cur);
+            cur = want;
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
+            T other[E];
+#pragma unroll
+            for (int r = 0; r < E; ++r) other[r] = Ops::shfl_xor(v[E - 1 - r], lane_mask);
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], Ops::reverse(other[r]));
+        }
+#pragma unroll
+        for (int j = k >> 2; j > 0; j >>= 1) {
             if (j < E) {
+                if (k > E && j == E / 2) {                // back to plain keys before the register stages
+#pragma unroll
+                    for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+                    cur = Ops::identity();
+                }
 #pragma unroll
                 for (int r = 0; r < E; ++r) {
                     if ((r & j) == 0) {
-                        const bool up = (k < E) ? ((r & k) == 0) : (((lane * E) & k) == 0);
                         const T a = v[r], b = v[r | j];
-                        const T lo = Ops::lo(a, b), hi = Ops::hi(a, b);
-                        v[r] = up ? lo : hi;
-                        v[r | j] = up ? hi : lo;
+                        v[r] = Ops::lo(a, b);
+                        v[r | j] = Ops::hi(a, b);
                     }
                 }
             } else {
                 const int lane_mask = j / E;
-                const bool lower = (lane & lane_mask) == 0;
-                const bool up = ((lane * E) & k) == 0;
-                const bool keep_lo = (lower == up);
+                const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
+                const typename Ops::Flip f = Ops::combine(want, cur);
+                cur = want;
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
 #pragma unroll
                 for (int r = 0; r < E; ++r) {
                     const T other = Ops::shfl_xor(v[r], lane_mask);
-                    v[r] = keep_lo ? Ops::lo(v[r], other) : Ops::hi(v[r], other);
+                    v[r] = Ops::lo(v[r], Ops::reverse(other));
                 }
             }
         }
     }
+    if (E == 1) v[0] = Ops::apply(v[0], cur);             // no register stage ever undid the reversal
 }
 
 // Bitonic sorting network over P keys (a power of two) in shared memory, all threads of the CTA.
@@ -113,6 +164,100 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_warp(const float* 
         float s = 0.0f;
 #pragma unroll
         for (int w = 0; w < kSortWarps; ++w) s += stage[w][j];
+        partial[static_cast<size_t>(blockIdx.x) * N + j] = s;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same, with the rows brought into shared memory by the bulk-copy engine one row ahead of the
+// sort: each warp owns two row buffers and two mbarriers; while it sorts row i, row i+1 is in
+// flight, so the sort never waits on global memory.  Needs ldx*4 and the matrix base to be
+// multiples of 16 bytes.  Dynamic shared memory: kSortWarps * 2 * ldx floats (reused for the CTA
+// reduction at the end), then 2 * kSortWarps mbarriers and the abort flag.
+// ---------------------------------------------------------------------------------------------
+template <int E>
+inline size_t sort_tma_smem_bytes(int ldx) {
+    const size_t rows = static_cast<size_t>(kSortWarps) * 2 * ldx * sizeof(float);
+    const size_t stage = static_cast<size_t>(kSortWarps) * 32 * E * sizeof(float);
+    return (rows > stage ? rows : stage) + 16 * kSortWarps + 16;
+}
+
+template <int E>
+__global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* __restrict__ x, int ldx, int N, int count,
+                                                                   float* __restrict__ partial, DevState* st) {
+    using namespace cutoff::async;
+    extern __shared__ __align__(16) float sm_sort[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t row_floats = static_cast<size_t>(kSortWarps) * 2 * ldx;
+    const size_t stage_floats = static_cast<size_t>(kSortWarps) * 32 * E;
+    const size_t data_floats = row_floats > stage_floats ? row_floats : stage_floats;
+    const uint32_t bars = smem_u32(sm_sort + data_floats);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm_sort + data_floats + 4 * kSortWarps);
+    float* const buf0 = sm_sort + static_cast<size_t>(warp) * 2 * ldx;      // buffer b = buf0 + b*ldx
+    const uint32_t bar0 = bars + 16u * warp;                                // barrier b = bar0 + 8*b
+    const uint32_t row_bytes = static_cast<uint32_t>(ldx) * 4u;
+    if (threadIdx.x == 0) *abort_flag = 0;
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8u, 1);
+        fence_barrier_init();
+        fence_proxy_async();
+    }
+    __syncthreads();
+
+    float acc[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) acc[r] = 0.0f;
+    const int stride = gridDim.x * kSortWarps;
+    int row = blockIdx.x * kSortWarps + warp;
+    if (row < count && lane == 0) {
+        mbar_arrive_expect_tx(bar0, row_bytes);
+        bulk_load_1d(smem_u32(buf0), x + static_cast<size_t>(row) * ldx, row_bytes, bar0);
+    }
+    bool aborted = false;
+    // iteration `it` uses buffer it & 1 for the (it >> 1)-th time: its barrier completes phase (it >> 1) & 1
+    for (uint32_t it = 0; row < count; row += stride, ++it) {
+        const uint32_t b = it & 1u, par = (it >> 1) & 1u;
+        const int next = row + stride;
+        if (next < count) {
+            // the other buffer was read in the previous iteration: order those reads before the engine's write
+            fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+                const uint32_t nb = b ^ 1u;
+                mbar_arrive_expect_tx(bar0 + 8u * nb, row_bytes);
+                bulk_load_1d(smem_u32(buf0 + nb * ldx), x + static_cast<size_t>(next) * ldx, row_bytes, bar0 + 8u * nb);
+            }
+        }
+        if (!mbar_wait(bar0 + 8u * b, par, abort_flag, st)) {
+            // wind down: give both copies that may still be in flight time to land (bounded)
+            mbar_wait_quiet(bar0 + 8u * b, par);
+            if (next < count) mbar_wait_quiet(bar0 + 8u * (b ^ 1u), ((it + 1u) >> 1) & 1u);
+            aborted = true;
+            break;
+        }
+        const float* src = buf0 + b * ldx;
+        float v[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int e = r * 32 + lane;
+            v[r] = e < N ? src[e] : INFINITY;
+        }
+        __syncwarp();
+        warp_bitonic_sort<float, E>(v, lane);
+#pragma unroll
+        for (int r = 0; r < E; ++r) acc[r] += v[r];
+    }
+    (void)aborted;
+    __syncthreads();                                   // all row buffers are dead: reuse them as the stage
+    float* stage = sm_sort;
+#pragma unroll
+    for (int r = 0; r < E; ++r) stage[warp * 32 * E + lane * E + r] = acc[r];
+    __syncthreads();
+    for (int j = threadIdx.x; j < N; j += kSortWarps * 32) {
+        float s = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kSortWarps; ++w) s += stage[w * 32 * E + j];
         partial[static_cast<size_t>(blockIdx.x) * N + j] = s;
     }
 }

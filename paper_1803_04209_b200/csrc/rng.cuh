@@ -47,12 +47,40 @@ __device__ __forceinline__ void box_muller(uint32_t r_a, uint32_t r_b, float& e_
     e_sin = radius * s;
 }
 
+// The same transform with the hardware approximations (lg2, sqrt, sin, cos): each is accurate to
+// about 1e-6 absolute on the ranges used here, except that sqrt(-2 ln u1) loses relative accuracy
+// for the rare u1 within ~1e-3 of 1 (radius below ~0.05, absolute error still below ~6e-4).
+// Used only where the surrounding arithmetic is tf32.  The angle is taken in [-pi, pi) -- the same
+// point on the circle as 2 pi u2 -- where the sine / cosine units are most accurate.
+__device__ __forceinline__ void box_muller_fast(uint32_t r_a, uint32_t r_b, float& e_cos, float& e_sin) {
+    const float u1 = static_cast<float>((r_a >> 8) + 1u) * 0x1p-24f;
+    const float angle = static_cast<float>(static_cast<int32_t>(r_b) >> 8) * (6.283185307179586f * 0x1p-24f);
+    const float r2 = fmaxf(-1.3862943611198906f * __log2f(u1), 0.0f);     // -2 ln u1
+    float radius;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(r2));
+    e_cos = radius * __cosf(angle);
+    e_sin = radius * __sinf(angle);
+}
+
+__device__ __forceinline__ float exp_half_fast(float logvar) {            // exp(logvar / 2)
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(logvar * 0.7213475204444817f));
+    return r;
+}
+
 // Four standard normals for elements 4q..4q+3.
 __device__ __forceinline__ void normal4(uint32_t q, uint32_t sample, uint32_t stream, uint32_t step,
                                         uint32_t seed_lo, uint32_t seed_hi, float out[4]) {
     const Philox4 r = philox4x32_10(q, sample, stream, step, seed_lo, seed_hi);
     box_muller(r.x, r.y, out[0], out[1]);
     box_muller(r.z, r.w, out[2], out[3]);
+}
+
+__device__ __forceinline__ void normal4_fast(uint32_t q, uint32_t sample, uint32_t stream, uint32_t step,
+                                             uint32_t seed_lo, uint32_t seed_hi, float out[4]) {
+    const Philox4 r = philox4x32_10(q, sample, stream, step, seed_lo, seed_hi);
+    box_muller_fast(r.x, r.y, out[0], out[1]);
+    box_muller_fast(r.z, r.w, out[2], out[3]);
 }
 
 }  // namespace cutoff
