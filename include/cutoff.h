@@ -77,7 +77,7 @@ enum {
 typedef struct {
     int32_t n_workers;          /* N >= 1                                                          */
     int32_t latent_dim;         /* D in {4, 8, 16, 32}                                             */
-    int32_t hidden;             /* H, multiple of 4 (multiple of 32 for the tensor-core precisions) */
+    int32_t hidden;             /* H, a multiple of D (and so of 4)                                */
     int32_t lag;                /* the paper's l >= 0; the window holds l+1 vectors                */
     int32_t n_samples;          /* S: samples this context draws per decision (the paper's K)      */
     int32_t precision;          /* CUTOFF_PRECISION_*                                              */

@@ -27,12 +27,12 @@ struct ModelDev {
     int N, D, H, W;          // workers, latent size, hidden width, window = lag + 1
     // encoder RNNs
     const float *Wxf, *Whf, *bf, *a0, *Wxb, *Whb, *bb, *b0;
-    // guide
-    const float *Wz, *bz, *WmuT /*[H x D]*/, *bmu, *Wsig, *bsig, *z0;
-    // transition
-    const float *W1, *b1, *W2T /*[H x 2D]*/, *b2;
-    // emission
-    const float *W3, *b3, *W4 /*[2N x H]*/, *b4;
+    // guide (WzT is the transposed copy [D x H]; Wmu as loaded [D x H])
+    const float *WzT, *bz, *Wmu, *bmu, *Wsig, *bsig, *z0;
+    // transition (W1T transposed copy [D x H]; W2 as loaded [2D x H])
+    const float *W1T, *b1, *W2, *b2;
+    // emission (W3T transposed copy [D x H]; W4 as loaded [2N x H])
+    const float *W3T, *b3, *W4, *b4;
 };
 
 struct NoiseKey {

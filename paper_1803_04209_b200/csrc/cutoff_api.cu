@@ -38,8 +38,7 @@ struct cutoff_ctx {
     cudaStream_t stream = nullptr;
 
     float* d_blob = nullptr;        // tensors as loaded
-    float* d_WmuT = nullptr;        // [H][D]
-    float* d_W2T = nullptr;         // [H][2D]
+    float* d_WT = nullptr;          // transposed copies WzT, W1T, W3T: 3 x [D][H]
     ModelDev m{};
     bool weights_loaded = false;
 
@@ -105,7 +104,7 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
-    cudaFree(c->d_blob); cudaFree(c->d_WmuT); cudaFree(c->d_W2T); cudaFree(c->d_ring); cudaFree(c->d_stage);
+    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
     cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
     if (c->h_stage) cudaFreeHost(c->h_stage);
@@ -169,11 +168,23 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
     static bool attr_set = false;
     if (!attr_set) {
         cudaFuncSetAttribute(k_chain<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        cudaFuncSetAttribute(k_chain_resident<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
         attr_set = true;
     }
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
-    k_chain<D><<<ceil_div(count, kChainThreads / (D / 4)), kChainThreads, smem, c->stream>>>(
-        c->m, c->d_hlr, c->d_state, key, sample_base, count, c->cfg.precision != CUTOFF_PRECISION_FP32, c->d_v);
+    const int round_v = c->cfg.precision != CUTOFF_PRECISION_FP32;
+    const size_t resident = chain_resident_smem_floats(c->D, c->H, c->W) * sizeof(float);
+    if (resident <= 200 * 1024) {
+        // all weights fit: one persistent CTA per SM, as many as there are warp batches to hand out
+        const int batch = 32 / ChainShape<D>::G * ChainShape<D>::SPL;
+        const int ctas_needed = ceil_div(ceil_div(count, batch), kChainResidentThreads / 32);
+        const int grid = ctas_needed < c->sm_count ? ctas_needed : c->sm_count;
+        k_chain_resident<D><<<grid, kChainResidentThreads, resident, c->stream>>>(c->m, c->d_hlr, c->d_state, key,
+                                                                                sample_base, count, round_v, c->d_v);
+    } else {
+        k_chain<D><<<ceil_div(count, ChainShape<D>::kSamplesPerCta), kChainThreads, smem, c->stream>>>(
+            c->m, c->d_hlr, c->d_state, key, sample_base, count, round_v, c->d_v);
+    }
 }
 
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
@@ -343,7 +354,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
         cfg->total_samples < 0 || cfg->device < 0)
         return CUTOFF_ERR_BAD_ARG;
     if (cfg->precision < CUTOFF_PRECISION_FP32 || cfg->precision > CUTOFF_PRECISION_BF16W) return CUTOFF_ERR_BAD_ARG;
-    if (!valid_latent(cfg->latent_dim) || cfg->hidden % 4 != 0) return CUTOFF_ERR_UNSUPPORTED;
+    if (!valid_latent(cfg->latent_dim) || cfg->hidden % cfg->latent_dim != 0) return CUTOFF_ERR_UNSUPPORTED;
     if (cfg->n_workers > 4096 || cfg->hidden > 1024 || cfg->lag > 255) return CUTOFF_ERR_UNSUPPORTED;
     if (cfg->sample_offset + cfg->n_samples > (1ll << 32)) return CUTOFF_ERR_UNSUPPORTED;
     if (cfg->total_samples > 0 && cfg->total_samples < cfg->n_samples) return CUTOFF_ERR_BAD_ARG;
@@ -381,8 +392,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     size_t blob_floats = 0;
     for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
     CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
-    CREATE_CHECK(cudaMalloc(&c->d_WmuT, sizeof(float) * c->H * c->D));
-    CREATE_CHECK(cudaMalloc(&c->d_W2T, sizeof(float) * c->H * 2 * c->D));
+    CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 3 * c->H * c->D));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_state, sizeof(DevState)));
@@ -454,27 +464,26 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         }
     }
     CU_CHECK(c, cudaMemcpy(c->d_blob, host.data(), total * sizeof(float), cudaMemcpyHostToDevice));
-    // transposed copies for the per-sample chain
+    // transposed copies [D][H] of the three latent-to-hidden matrices for the per-sample chain
     const size_t D = c->D, H = c->H;
-    std::vector<float> wmuT(H * D), w2T(H * 2 * D);
-    const float* wmu = host.data() + off[10];
-    const float* w2 = host.data() + off[17];
-    for (size_t d = 0; d < D; ++d)
-        for (size_t i = 0; i < H; ++i) wmuT[i * D + d] = wmu[d * H + i];
-    for (size_t r = 0; r < 2 * D; ++r)
-        for (size_t i = 0; i < H; ++i) w2T[i * 2 * D + r] = w2[r * H + i];
-    CU_CHECK(c, cudaMemcpy(c->d_WmuT, wmuT.data(), wmuT.size() * sizeof(float), cudaMemcpyHostToDevice));
-    CU_CHECK(c, cudaMemcpy(c->d_W2T, w2T.data(), w2T.size() * sizeof(float), cudaMemcpyHostToDevice));
+    std::vector<float> wT(3 * H * D);
+    const size_t src_off[3] = {off[8], off[15], off[19]};           // Wz, W1, W3: each [H][D]
+    for (int t = 0; t < 3; ++t) {
+        const float* w = host.data() + src_off[t];
+        for (size_t i = 0; i < H; ++i)
+            for (size_t d = 0; d < D; ++d) wT[t * H * D + d * H + i] = w[i * D + d];
+    }
+    CU_CHECK(c, cudaMemcpy(c->d_WT, wT.data(), wT.size() * sizeof(float), cudaMemcpyHostToDevice));
 
     ModelDev& m = c->m;
     m.N = c->N; m.D = c->D; m.H = c->H; m.W = c->W;
     const float* b = c->d_blob;
     m.Wxf = b + off[0]; m.Whf = b + off[1]; m.bf = b + off[2]; m.a0 = b + off[3];
     m.Wxb = b + off[4]; m.Whb = b + off[5]; m.bb = b + off[6]; m.b0 = b + off[7];
-    m.Wz = b + off[8]; m.bz = b + off[9]; m.WmuT = c->d_WmuT; m.bmu = b + off[11];
+    m.WzT = c->d_WT; m.bz = b + off[9]; m.Wmu = b + off[10]; m.bmu = b + off[11];
     m.Wsig = b + off[12]; m.bsig = b + off[13]; m.z0 = b + off[14];
-    m.W1 = b + off[15]; m.b1 = b + off[16]; m.W2T = c->d_W2T; m.b2 = b + off[18];
-    m.W3 = b + off[19]; m.b3 = b + off[20]; m.W4 = b + off[21]; m.b4 = b + off[22];
+    m.W1T = c->d_WT + H * D; m.b1 = b + off[16]; m.W2 = b + off[17]; m.b2 = b + off[18];
+    m.W3T = c->d_WT + 2 * H * D; m.b3 = b + off[20]; m.W4 = b + off[21]; m.b4 = b + off[22];
     if (c->use_tc) {
         const int rc = make_tile_map(c, &c->map_w4, m.W4, 2ull * c->N, static_cast<uint64_t>(c->H));
         if (rc) return rc;

@@ -138,16 +138,34 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
 // ---------------------------------------------------------------------------------------------
 // Per-sample chain: guide steps over the window, transition, first emission layer.
 //
-// A sample is worked on by a group of G = D/4 adjacent lanes.  Lane g of the group owns the hidden
-// units i = g, g+G, g+2G, ... of every layer and the four latent dimensions 4g..4g+3 (exactly one
-// Philox call per noise stream).  Every lane keeps the whole latent vector in registers; partial
-// layer outputs are summed over the group with xor-shuffles.  Weights are staged in shared memory
-// phase by phase, rows padded by four floats so that the G rows a warp reads at once fall into
-// different banks.
+// SPL samples are worked on by a group of G = D/4 adjacent lanes.  Lane g of the group owns, of
+// every hidden layer, the units i = 4(g + G m) .. 4(g + G m) + 3 (m = 0, 1, ...) and the four
+// latent dimensions 4g..4g+3 (exactly one Philox call per noise stream and sample).  Every lane
+// keeps the whole latent vector of its samples in registers.  A layer pair
+//      hidden = act(A z + a),   out += B hidden
+// is evaluated four hidden units at a time as two small outer-product updates: A is staged
+// transposed ([D][H]) and B as it is ([out][H]), so that the four weights a lane needs for one
+// input or output dimension are one 16-byte shared-memory load, which the G lanes of a group read
+// from consecutive addresses and all groups of a warp read as a broadcast.  Partial outputs are
+// summed over the group with xor-shuffles.  Each weight read serves all SPL samples of the lane.
 // ---------------------------------------------------------------------------------------------
-constexpr int kChainThreads = 256;
+constexpr int kChainThreads = 128;
+
+template <int D> struct ChainShape {
+    static constexpr int G = D / 4;                   // lanes per group
+    static constexpr int SPL = D <= 16 ? 2 : 1;       // samples per lane
+    static constexpr int kSamplesPerCta = kChainThreads / G * SPL;
+};
 
 __device__ __forceinline__ float softplusf(float x) { return x > 20.0f ? x : log1pf(expf(x)); }
+
+// tanh(x) = 1 - 2 / (exp(2x) + 1) with the hardware exp2 and reciprocal: absolute error below 3e-7.
+__device__ __forceinline__ float tanh_fast(float x) {
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 2.8853900817779268f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return fmaf(-2.0f, r, 1.0f);
+}
 
 __device__ __forceinline__ float round_tf32(float x) {
     uint32_t r;
@@ -155,38 +173,42 @@ __device__ __forceinline__ float round_tf32(float x) {
     return __uint_as_float(r);
 }
 
-// Copy a row-major [rows][cols] matrix into shared memory with row stride ld.
-__device__ __forceinline__ void stage_matrix(float* dst, const float* __restrict__ src, int rows, int cols, int ld) {
-    for (int idx = threadIdx.x; idx < rows * cols; idx += blockDim.x) {
-        const int r = idx / cols, c = idx - r * cols;
-        dst[r * ld + c] = src[idx];
+__device__ __forceinline__ void stage_vector(float* dst, const float* __restrict__ src, int n) {
+    for (int i = threadIdx.x; i < n; i += blockDim.x) dst[i] = src[i];
+}
+
+__device__ __forceinline__ float4 lds4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+
+// hidden[s][c] = sum_k A^T[k][i0 + c] * z[s][k] + bias[i0 + c]       (A^T staged as [D][H])
+template <int D, int SPL>
+__device__ __forceinline__ void hidden_block(const float* sAT, const float* sbias, int H, int i0,
+                                             const float (&z)[SPL][D], float (&hid)[SPL][4]) {
+    const float4 b = lds4(sbias + i0);
+#pragma unroll
+    for (int s = 0; s < SPL; ++s) { hid[s][0] = b.x; hid[s][1] = b.y; hid[s][2] = b.z; hid[s][3] = b.w; }
+#pragma unroll
+    for (int k = 0; k < D; ++k) {
+        const float4 w = lds4(sAT + k * H + i0);
+#pragma unroll
+        for (int s = 0; s < SPL; ++s) {
+            hid[s][0] = fmaf(w.x, z[s][k], hid[s][0]);
+            hid[s][1] = fmaf(w.y, z[s][k], hid[s][1]);
+            hid[s][2] = fmaf(w.z, z[s][k], hid[s][2]);
+            hid[s][3] = fmaf(w.w, z[s][k], hid[s][3]);
+        }
     }
 }
 
-template <int D>
-__device__ __forceinline__ float dot_smem(const float* w, const float (&z)[D], float acc) {
-    const float4* w4 = reinterpret_cast<const float4*>(w);
+// out[s][o] += sum_c B[o][i0 + c] * hid[s][c]                        (B staged as [M][H])
+template <int M, int SPL>
+__device__ __forceinline__ void output_block(const float* sB, int H, int i0, const float (&hid)[SPL][4],
+                                             float (&out)[SPL][M]) {
 #pragma unroll
-    for (int d4 = 0; d4 < D / 4; ++d4) {
-        const float4 q = w4[d4];
-        acc = fmaf(q.x, z[4 * d4 + 0], acc);
-        acc = fmaf(q.y, z[4 * d4 + 1], acc);
-        acc = fmaf(q.z, z[4 * d4 + 2], acc);
-        acc = fmaf(q.w, z[4 * d4 + 3], acc);
-    }
-    return acc;
-}
-
-template <int D2>
-__device__ __forceinline__ void axpy_smem(const float* w, float a, float (&y)[D2]) {
-    const float4* w4 = reinterpret_cast<const float4*>(w);
+    for (int o = 0; o < M; ++o) {
+        const float4 w = lds4(sB + o * H + i0);
 #pragma unroll
-    for (int d4 = 0; d4 < D2 / 4; ++d4) {
-        const float4 q = w4[d4];
-        y[4 * d4 + 0] = fmaf(q.x, a, y[4 * d4 + 0]);
-        y[4 * d4 + 1] = fmaf(q.y, a, y[4 * d4 + 1]);
-        y[4 * d4 + 2] = fmaf(q.z, a, y[4 * d4 + 2]);
-        y[4 * d4 + 3] = fmaf(q.w, a, y[4 * d4 + 3]);
+        for (int s = 0; s < SPL; ++s)
+            out[s][o] = fmaf(w.w, hid[s][3], fmaf(w.z, hid[s][2], fmaf(w.y, hid[s][1], fmaf(w.x, hid[s][0], out[s][o]))));
     }
 }
 
@@ -220,114 +242,242 @@ __device__ __forceinline__ void group_allgather(const float (&own)[4], float (&z
 
 // Shared memory needed by k_chain, in floats.
 inline size_t chain_smem_floats(int D, int H, int W) {
-    const size_t ld = D + 4, ld2 = 2 * D + 4;
-    const size_t guide = 2 * H * ld + H + static_cast<size_t>(W) * H + D * ld;
-    const size_t trans = H * ld + H * ld2 + H;
+    const size_t guide = 2 * static_cast<size_t>(H) * D + H + static_cast<size_t>(W) * H + static_cast<size_t>(D) * D;
+    const size_t trans = 3 * static_cast<size_t>(H) * D + H;
     return guide > trans ? guide : trans;
 }
 
+__device__ __forceinline__ void stage_vector4(float* dst, const float* __restrict__ src, int n) {   // n % 4 == 0
+    const float4* s4 = reinterpret_cast<const float4*>(src);
+    float4* d4 = reinterpret_cast<float4*>(dst);
+    for (int i = threadIdx.x; i < n / 4; i += blockDim.x) d4[i] = s4[i];
+}
+
+struct ChainNoise {
+    NoiseKey key;
+    uint32_t step;
+    uint32_t sample0;          // global index of the lane's first sample
+};
+
+// Guide: z_t = mu + sigma * eps for t = 0..W-1 (Section 3.1.3).  z holds z_{T-l-1} on entry, z_T on exit.
 template <int D>
-__global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float* __restrict__ hlr,
-                                                          const DevState* __restrict__ st, NoiseKey key,
-                                                          uint32_t sample_base, int count, int round_v,
-                                                          float* __restrict__ v_out /*[count][H]*/) {
-    constexpr int G = D / 4, LD = D + 4, LD2 = 2 * D + 4;
-    extern __shared__ __align__(16) float sm[];
+__device__ __forceinline__ void chain_guide(const ModelDev& m, const float* sWzT, const float* sWmu, const float* sWsig,
+                                            const float* sbz, const float* shl, int g, const ChainNoise& nz,
+                                            float (&z)[ChainShape<D>::SPL][D]) {
+    constexpr int G = ChainShape<D>::G, SPL = ChainShape<D>::SPL;
     const int H = m.H, W = m.W;
-    const int g = threadIdx.x % G;
-    const int k = blockIdx.x * (kChainThreads / G) + threadIdx.x / G;
-    const uint32_t sample = sample_base + static_cast<uint32_t>(k);
-    const uint32_t step = st->step;
-
-    // ---- guide: z_t = mu + sigma * eps over the window --------------------------------------
-    float* sWz = sm;                    // [H][LD]
-    float* sWmuT = sWz + H * LD;        // [H][LD]
-    float* sWsig = sWmuT + H * LD;      // [D][LD]
-    float* sbz = sWsig + D * LD;        // [H]
-    float* shl = sbz + H;               // [W][H]  h_left + h_right
-    stage_matrix(sWz, m.Wz, H, D, LD);
-    stage_matrix(sWmuT, m.WmuT, H, D, LD);
-    stage_matrix(sWsig, m.Wsig, D, D, LD);
-    for (int i = threadIdx.x; i < H; i += kChainThreads) sbz[i] = m.bz[i];
-    for (int i = threadIdx.x; i < W * H; i += kChainThreads) shl[i] = hlr[i] + hlr[W * H + i];
-    __syncthreads();
-
-    float z[D];
-#pragma unroll
-    for (int d = 0; d < D; ++d) z[d] = m.z0[d];
     for (int t = 0; t < W; ++t) {
-        float mu[D];
+        float mu[SPL][D];
 #pragma unroll
-        for (int d = 0; d < D; ++d) mu[d] = 0.0f;
+        for (int s = 0; s < SPL; ++s)
+#pragma unroll
+            for (int d = 0; d < D; ++d) mu[s][d] = 0.0f;
         const float* hl = shl + t * H;
-#pragma unroll 2
-        for (int i = g; i < H; i += G) {
-            const float pre = dot_smem<D>(sWz + i * LD, z, sbz[i]);
-            const float h_out = (tanhf(pre) + hl[i]) * (1.0f / 3.0f);
-            axpy_smem<D>(sWmuT + i * LD, h_out, mu);
-        }
-        group_allreduce<G, D>(mu);
+        for (int i0 = 4 * g; i0 < H; i0 += 4 * G) {
+            float hid[SPL][4];
+            hidden_block<D, SPL>(sWzT, sbz, H, i0, z, hid);
+            const float4 lr = lds4(hl + i0);
+            const float lrv[4] = {lr.x, lr.y, lr.z, lr.w};
 #pragma unroll
-        for (int d = 0; d < D; ++d) mu[d] += m.bmu[d];
-        float eps[4], mu_own[4], z_own[4];
-        normal4(static_cast<uint32_t>(g), sample, static_cast<uint32_t>(t), step, key.seed_lo, key.seed_hi, eps);
-        select_own<G, D>(mu, 0, g, mu_own);
+            for (int s = 0; s < SPL; ++s)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const int d = 4 * g + c;
-            const float pre = dot_smem<D>(sWsig + d * LD, mu, m.bsig[d]);
-            z_own[c] = fmaf(softplusf(pre), eps[c], mu_own[c]);
+                for (int c = 0; c < 4; ++c) hid[s][c] = (tanh_fast(hid[s][c]) + lrv[c]) * (1.0f / 3.0f);
+            output_block<D, SPL>(sWmu, H, i0, hid, mu);
         }
-        group_allgather<G, D>(z_own, z);
+#pragma unroll
+        for (int s = 0; s < SPL; ++s) {
+            group_allreduce<G, D>(mu[s]);
+#pragma unroll
+            for (int d = 0; d < D; ++d) mu[s][d] += m.bmu[d];
+        }
+#pragma unroll
+        for (int s = 0; s < SPL; ++s) {
+            float eps[4], mu_own[4], z_own[4];
+            normal4(static_cast<uint32_t>(g), nz.sample0 + s, static_cast<uint32_t>(t), nz.step, nz.key.seed_lo,
+                    nz.key.seed_hi, eps);
+            select_own<G, D>(mu[s], 0, g, mu_own);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float pre = m.bsig[4 * g + c];
+                const float* wrow = sWsig + (4 * g + c) * D;
+#pragma unroll
+                for (int e4 = 0; e4 < D / 4; ++e4) {
+                    const float4 w = lds4(wrow + 4 * e4);
+                    pre = fmaf(w.x, mu[s][4 * e4 + 0], pre);
+                    pre = fmaf(w.y, mu[s][4 * e4 + 1], pre);
+                    pre = fmaf(w.z, mu[s][4 * e4 + 2], pre);
+                    pre = fmaf(w.w, mu[s][4 * e4 + 3], pre);
+                }
+                z_own[c] = fmaf(softplusf(pre), eps[c], mu_own[c]);
+            }
+            group_allgather<G, D>(z_own, z[s]);
+        }
     }
-    __syncthreads();
+}
 
-    // ---- transition: z_{T+1} = mean + exp(logvar / 2) * eps ---------------------------------
-    float* sW1 = sm;                    // [H][LD]
-    float* sW2T = sW1 + H * LD;         // [H][LD2]
-    float* sb1 = sW2T + H * LD2;        // [H]
-    stage_matrix(sW1, m.W1, H, D, LD);
-    stage_matrix(sW2T, m.W2T, H, 2 * D, LD2);
-    for (int i = threadIdx.x; i < H; i += kChainThreads) sb1[i] = m.b1[i];
-    __syncthreads();
-    {
-        float head[2 * D];
+// Transition: z_{T+1} = mean + exp(logvar / 2) * eps with [mean | logvar] = W2 relu(W1 z + b1) + b2.
+template <int D>
+__device__ __forceinline__ void chain_transition(const ModelDev& m, const float* sW1T, const float* sW2, const float* sb1,
+                                                 int g, const ChainNoise& nz, float (&z)[ChainShape<D>::SPL][D]) {
+    constexpr int G = ChainShape<D>::G, SPL = ChainShape<D>::SPL;
+    const int H = m.H;
+    float head[SPL][2 * D];
 #pragma unroll
-        for (int o = 0; o < 2 * D; ++o) head[o] = 0.0f;
-#pragma unroll 2
-        for (int i = g; i < H; i += G) {
-            const float u = fmaxf(dot_smem<D>(sW1 + i * LD, z, sb1[i]), 0.0f);
-            axpy_smem<2 * D>(sW2T + i * LD2, u, head);
-        }
-        group_allreduce<G, 2 * D>(head);
+    for (int s = 0; s < SPL; ++s)
+#pragma unroll
+        for (int o = 0; o < 2 * D; ++o) head[s][o] = 0.0f;
+    for (int i0 = 4 * g; i0 < H; i0 += 4 * G) {
+        float hid[SPL][4];
+        hidden_block<D, SPL>(sW1T, sb1, H, i0, z, hid);
+#pragma unroll
+        for (int s = 0; s < SPL; ++s)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) hid[s][c] = fmaxf(hid[s][c], 0.0f);
+        output_block<2 * D, SPL>(sW2, H, i0, hid, head);
+    }
+#pragma unroll
+    for (int s = 0; s < SPL; ++s) {
+        group_allreduce<G, 2 * D>(head[s]);
         float eps[4], mean_own[4], logvar_own[4], z_own[4];
-        normal4(static_cast<uint32_t>(g), sample, kStreamTransition, step, key.seed_lo, key.seed_hi, eps);
-        select_own<G, 2 * D>(head, 0, g, mean_own);
-        select_own<G, 2 * D>(head, D, g, logvar_own);
+        normal4(static_cast<uint32_t>(g), nz.sample0 + s, kStreamTransition, nz.step, nz.key.seed_lo, nz.key.seed_hi, eps);
+        select_own<G, 2 * D>(head[s], 0, g, mean_own);
+        select_own<G, 2 * D>(head[s], D, g, logvar_own);
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
             const float mean = mean_own[c] + m.b2[4 * g + c];
             const float logvar = logvar_own[c] + m.b2[D + 4 * g + c];
             z_own[c] = fmaf(expf(0.5f * logvar), eps[c], mean);
         }
-        group_allgather<G, D>(z_own, z);
+        group_allgather<G, D>(z_own, z[s]);
     }
+}
+
+// Emission hidden layer: v = relu(W3 z + b3), written for the samples k0 .. k0+SPL-1 that exist.
+template <int D>
+__device__ __forceinline__ void chain_emission_hidden(const ModelDev& m, const float* sW3T, const float* sb3, int g,
+                                                      const float (&z)[ChainShape<D>::SPL][D], int k0, int count,
+                                                      int round_v, float* __restrict__ v_out) {
+    constexpr int G = ChainShape<D>::G, SPL = ChainShape<D>::SPL;
+    const int H = m.H;
+    for (int i0 = 4 * g; i0 < H; i0 += 4 * G) {
+        float hid[SPL][4];
+        hidden_block<D, SPL>(sW3T, sb3, H, i0, z, hid);
+#pragma unroll
+        for (int s = 0; s < SPL; ++s) {
+            float4 o;
+            o.x = fmaxf(hid[s][0], 0.0f); o.y = fmaxf(hid[s][1], 0.0f);
+            o.z = fmaxf(hid[s][2], 0.0f); o.w = fmaxf(hid[s][3], 0.0f);
+            if (round_v) { o.x = round_tf32(o.x); o.y = round_tf32(o.y); o.z = round_tf32(o.z); o.w = round_tf32(o.w); }
+            if (k0 + s < count) *reinterpret_cast<float4*>(v_out + static_cast<size_t>(k0 + s) * H + i0) = o;
+        }
+    }
+}
+
+// Variant 1: weights staged phase by phase (any model size whose largest phase fits in shared memory).
+template <int D>
+__global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float* __restrict__ hlr,
+                                                          const DevState* __restrict__ st, NoiseKey key,
+                                                          uint32_t sample_base, int count, int round_v,
+                                                          float* __restrict__ v_out /*[count][H]*/) {
+    constexpr int G = ChainShape<D>::G, SPL = ChainShape<D>::SPL;
+    extern __shared__ __align__(16) float sm[];
+    const int H = m.H, W = m.W;
+    const int g = threadIdx.x % G;
+    const int k0 = (blockIdx.x * (kChainThreads / G) + threadIdx.x / G) * SPL;      // first sample of the lane
+    const ChainNoise nz{key, st->step, sample_base + static_cast<uint32_t>(k0)};
+
+    float* sWzT = sm;                   // [D][H]
+    float* sWmu = sWzT + H * D;         // [D][H]
+    float* sWsig = sWmu + H * D;        // [D][D]
+    float* sbz = sWsig + D * D;         // [H]
+    float* shl = sbz + H;               // [W][H]  h_left + h_right
+    stage_vector4(sWzT, m.WzT, H * D);
+    stage_vector4(sWmu, m.Wmu, H * D);
+    stage_vector4(sWsig, m.Wsig, D * D);
+    stage_vector4(sbz, m.bz, H);
+    for (int i = threadIdx.x; i < W * H; i += kChainThreads) shl[i] = hlr[i] + hlr[W * H + i];
+    __syncthreads();
+    float z[SPL][D];
+#pragma unroll
+    for (int s = 0; s < SPL; ++s)
+#pragma unroll
+        for (int d = 0; d < D; ++d) z[s][d] = m.z0[d];
+    chain_guide<D>(m, sWzT, sWmu, sWsig, sbz, shl, g, nz, z);
     __syncthreads();
 
-    // ---- emission, hidden layer: v = relu(W3 z + b3) ----------------------------------------
-    float* sW3 = sm;                    // [H][LD]
-    float* sb3 = sW3 + H * LD;          // [H]
-    stage_matrix(sW3, m.W3, H, D, LD);
-    for (int i = threadIdx.x; i < H; i += kChainThreads) sb3[i] = m.b3[i];
+    float* sW1T = sm;                   // [D][H]
+    float* sW2 = sW1T + H * D;          // [2D][H]
+    float* sb1 = sW2 + 2 * H * D;       // [H]
+    stage_vector4(sW1T, m.W1T, H * D);
+    stage_vector4(sW2, m.W2, 2 * H * D);
+    stage_vector4(sb1, m.b1, H);
     __syncthreads();
-    if (k < count) {
-        float* dst = v_out + static_cast<size_t>(k) * H;
-#pragma unroll 4
-        for (int i = g; i < H; i += G) {
-            float o = fmaxf(dot_smem<D>(sW3 + i * LD, z, sb3[i]), 0.0f);
-            if (round_v) o = round_tf32(o);
-            dst[i] = o;
-        }
+    chain_transition<D>(m, sW1T, sW2, sb1, g, nz, z);
+    __syncthreads();
+
+    float* sW3T = sm;                   // [D][H]
+    float* sb3 = sW3T + H * D;          // [H]
+    stage_vector4(sW3T, m.W3T, H * D);
+    stage_vector4(sb3, m.b3, H);
+    __syncthreads();
+    chain_emission_hidden<D>(m, sW3T, sb3, g, z, k0, count, round_v, v_out);
+}
+
+// Variant 2: every weight of the chain resident in shared memory, one persistent CTA per SM.
+// The weights are staged once; after that the warps never synchronise: warp w of the grid takes
+// the sample batches w, w + (warps in the grid), ... (a batch = the samples one warp covers).
+constexpr int kChainResidentThreads = 512;
+
+inline size_t chain_resident_smem_floats(int D, int H, int W) {
+    return 6 * static_cast<size_t>(H) * D + static_cast<size_t>(D) * D + 3 * static_cast<size_t>(H) +
+           static_cast<size_t>(W) * H;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kChainResidentThreads, 1)
+k_chain_resident(ModelDev m, const float* __restrict__ hlr, const DevState* __restrict__ st, NoiseKey key,
+                 uint32_t sample_base, int count, int round_v, float* __restrict__ v_out /*[count][H]*/) {
+    constexpr int G = ChainShape<D>::G, SPL = ChainShape<D>::SPL;
+    constexpr int kBatch = 32 / G * SPL;                // samples per warp and pass
+    extern __shared__ __align__(16) float sm[];
+    const int H = m.H, W = m.W;
+    float* sWzT = sm;                   // [D][H]
+    float* sWmu = sWzT + H * D;         // [D][H]
+    float* sW1T = sWmu + H * D;         // [D][H]
+    float* sW2 = sW1T + H * D;          // [2D][H]
+    float* sW3T = sW2 + 2 * H * D;      // [D][H]
+    float* sWsig = sW3T + H * D;        // [D][D]
+    float* sbz = sWsig + D * D;         // [H]
+    float* sb1 = sbz + H;               // [H]
+    float* sb3 = sb1 + H;               // [H]
+    float* shl = sb3 + H;               // [W][H]
+    stage_vector4(sWzT, m.WzT, H * D);
+    stage_vector4(sWmu, m.Wmu, H * D);
+    stage_vector4(sW1T, m.W1T, H * D);
+    stage_vector4(sW2, m.W2, 2 * H * D);
+    stage_vector4(sW3T, m.W3T, H * D);
+    stage_vector4(sWsig, m.Wsig, D * D);
+    stage_vector4(sbz, m.bz, H);
+    stage_vector4(sb1, m.b1, H);
+    stage_vector4(sb3, m.b3, H);
+    for (int i = threadIdx.x; i < W * H; i += kChainResidentThreads) shl[i] = hlr[i] + hlr[W * H + i];
+    __syncthreads();
+
+    const int lane = threadIdx.x & 31, g = lane % G;
+    const int warps_in_grid = gridDim.x * (kChainResidentThreads / 32);
+    const int n_batches = ceil_div(count, kBatch);
+    const uint32_t step = st->step;
+    for (int b = blockIdx.x * (kChainResidentThreads / 32) + (threadIdx.x >> 5); b < n_batches; b += warps_in_grid) {
+        const int k0 = b * kBatch + (lane / G) * SPL;
+        const ChainNoise nz{key, step, sample_base + static_cast<uint32_t>(k0)};
+        float z[SPL][D];
+#pragma unroll
+        for (int s = 0; s < SPL; ++s)
+#pragma unroll
+            for (int d = 0; d < D; ++d) z[s][d] = m.z0[d];
+        chain_guide<D>(m, sWzT, sWmu, sWsig, sbz, shl, g, nz, z);
+        chain_transition<D>(m, sW1T, sW2, sb1, g, nz, z);
+        chain_emission_hidden<D>(m, sW3T, sb3, g, z, k0, count, round_v, v_out);
     }
 }
 
