@@ -19,6 +19,8 @@ namespace {
 
 constexpr uint32_t kBlobMagic = 0x31465443u;   // "CTF1"
 constexpr int kNumStages = 5;
+constexpr int kMaxChunks = 64;        // passes per decision (also the number of timing event sets)
+constexpr int kPartialRows = 2048;    // partial-sum rows shared by all passes of a decision
 const char* const kStageNames[kNumStages] = {"encoder", "chain", "emission", "sort", "decide"};
 
 struct TensorSpec { const char* name; size_t rows, cols; };
@@ -67,7 +69,7 @@ struct cutoff_ctx {
     bool have_result = false;
 
     bool timing = false;
-    cudaEvent_t ev[kNumStages + 1][64]{};   // per chunk, stage boundaries
+    cudaEvent_t ev[kNumStages + 1][kMaxChunks]{};   // per chunk, stage boundaries
     bool ev_created = false;
     float stage_ms[kNumStages]{};
     int timed_chunks = 0;
@@ -121,16 +123,15 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
     int rows = chunk_rows_wanted > 0 ? chunk_rows_wanted : c->S;
     if (rows > c->S) rows = c->S;
     if (rows > c->alloc_rows) rows = c->alloc_rows;
+    if (ceil_div(c->S, rows) > kMaxChunks) rows = ceil_div(c->S, kMaxChunks);
     c->chunk_rows = rows;
     c->n_chunks = ceil_div(c->S, rows);
-    if (c->P <= 1024) {
-        const int want = ceil_div(rows, kSortWarps);
-        const int cap = c->sm_count * 2;
-        c->sort_grid = want < cap ? want : cap;
-    } else {
-        const int cap = c->sm_count * 2;
-        c->sort_grid = rows < cap ? rows : cap;
-    }
+    // CTAs of the sort kernel per pass: enough to fill the GPU, within the partial-sum rows available
+    int want, cap;
+    if (c->P <= 1024) { want = ceil_div(rows, kSortWarps); cap = c->sm_count * 2; }
+    else { want = rows; cap = c->sm_count * (c->P == 2048 ? 8 : 4); }
+    if (cap > kPartialRows / c->n_chunks) cap = kPartialRows / c->n_chunks;
+    c->sort_grid = want < cap ? want : cap;
 }
 
 template <int E>
@@ -153,9 +154,10 @@ int launch_sort(cutoff_ctx* c, int count, float* partial) {
         case 512: launch_sort_warp<16>(c, count, partial); break;
         case 1024: launch_sort_warp<32>(c, count, partial); break;
         case 2048:
+            k_sort_sum_cta<2><<<c->sort_grid, 64, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
+            break;
         case 4096:
-            k_sort_sum_cta<<<c->sort_grid, kSortCtaThreads, c->P * sizeof(float), c->stream>>>(
-                c->d_x, c->ldx, c->N, c->P, count, partial);
+            k_sort_sum_cta<4><<<c->sort_grid, 128, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
             break;
         default: return CUTOFF_ERR_UNSUPPORTED;
     }
@@ -270,7 +272,7 @@ int ensure_events(cutoff_ctx* c) {
 
 // Enqueue one decision's kernels.  advance = 1 for a real decision, 0 for the debug hook.
 int enqueue_decision(cutoff_ctx* c) {
-    const bool timed = c->timing && c->n_chunks <= 64;
+    const bool timed = c->timing;
     if (timed) {
         const int rc = ensure_events(c);
         if (rc) return rc;
@@ -386,6 +388,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
         if (cap < 1024) cap = 1024;
         c->alloc_rows = cap < c->S ? static_cast<int>(cap) : c->S;
     }
+    if (ceil_div(c->S, kMaxChunks) > c->alloc_rows) return fail(CUTOFF_ERR_UNSUPPORTED);   // S too large for the pass buffers
     plan_chunks(c, c->alloc_rows);
     c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
 
@@ -400,9 +403,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_hlr, sizeof(float) * 2 * c->W * c->H));
     CREATE_CHECK(cudaMalloc(&c->d_v, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->H));
     CREATE_CHECK(cudaMalloc(&c->d_x, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
-    // partial rows: room for the smallest allowed pass size (1024 rows)
-    const size_t max_partial_rows = static_cast<size_t>(ceil_div(c->S, 1024) + 1) * (c->sm_count * 2);
-    CREATE_CHECK(cudaMalloc(&c->d_partial, sizeof(float) * max_partial_rows * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_partial, sizeof(float) * static_cast<size_t>(kPartialRows) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_sums, sizeof(double) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_E, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_omega, sizeof(float) * c->N));
@@ -792,9 +793,8 @@ int cutoff_debug_sort(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t 
             case 256: k_debug_sort_warp<8><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
             case 512: k_debug_sort_warp<16><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
             case 1024: k_debug_sort_warp<32><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
-            default:
-                k_debug_sort_cta<<<grid_c, kSortCtaThreads, P * sizeof(unsigned long long), c->stream>>>(
-                    d_rows, n, P, rows_i, d_keys, d_perm);
+            case 2048: k_debug_sort_cta<2><<<grid_c, 64, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm); break;
+            default: k_debug_sort_cta<4><<<grid_c, 128, 0, c->stream>>>(d_rows, n, rows_i, d_keys, d_perm);
         }
         c->launches += 1;
         if (cudaMemcpyAsync(keys_out, d_keys, elems * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||

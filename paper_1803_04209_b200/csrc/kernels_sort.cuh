@@ -111,22 +111,87 @@ __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
     if (E == 1) v[0] = Ops::apply(v[0], cur);             // no register stage ever undid the reversal
 }
 
-// Bitonic sorting network over P keys (a power of two) in shared memory, all threads of the CTA.
-template <typename T>
-__device__ __forceinline__ void cta_bitonic_sort(T* s, int P) {
+// The half-cleaners idx <-> idx ^ j for j = 16E .. 1 of one merge, inside a warp: what remains of a
+// merge wider than the warp once its cross-warp exchanges are done.  Plain keys in, plain keys out.
+template <typename T, int E>
+__device__ __forceinline__ void warp_half_cleaners(T (&v)[E], int lane) {
     using Ops = KeyOps<T>;
-    for (int k = 2; k <= P; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int p = threadIdx.x; p < P / 2; p += blockDim.x) {
-                const int i = ((p & ~(j - 1)) << 1) | (p & (j - 1));      // index with bit j clear
-                const bool up = (i & k) == 0;
-                const T a = s[i], b = s[i | j];
-                const T lo = Ops::lo(a, b), hi = Ops::hi(a, b);
-                s[i] = up ? lo : hi;
-                s[i | j] = up ? hi : lo;
+    typename Ops::Flip cur = Ops::identity();
+#pragma unroll
+    for (int j = 16 * E; j >= E; j >>= 1) {
+        const int lane_mask = j / E;
+        const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
+        const typename Ops::Flip f = Ops::combine(want, cur);
+        cur = want;
+#pragma unroll
+        for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const T other = Ops::shfl_xor(v[r], lane_mask);
+            v[r] = Ops::lo(v[r], Ops::reverse(other));
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+#pragma unroll
+    for (int j = E / 2; j > 0; j >>= 1) {
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            if ((r & j) == 0) {
+                const T a = v[r], b = v[r | j];
+                v[r] = Ops::lo(a, b);
+                v[r | j] = Ops::hi(a, b);
+            }
+        }
+    }
+}
+
+// Bitonic sorting network over WPR * 1024 keys held by the WPR warps of a CTA, 32 keys per lane,
+// key index idx = (warp * 32 + lane) * 32 + r.  Each warp first sorts its 1024 keys in registers
+// and by shuffles; the merges of width 2048 and 4096 then start with exchanges between warps (one
+// for 2048, two for 4096), which go through shared memory (`xch`, WPR * 1024 keys, stored as
+// [register][thread] so that both the writes and the partner reads are conflict-free), and finish
+// inside the warps.  All threads of the CTA must call it.  Ascending on exit.
+template <typename T, int WPR>
+__device__ __forceinline__ void cta_bitonic_sort(T (&v)[32], T* xch) {
+    using Ops = KeyOps<T>;
+    constexpr int E = 32, T_ = WPR * 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    warp_bitonic_sort<T, E>(v, lane);
+#pragma unroll
+    for (int k = 2; k <= WPR; k <<= 1) {                 // merge width in warps
+        // mirror exchange: idx <-> idx ^ (k*1024 - 1)
+        {
+#pragma unroll
+            for (int r = 0; r < E; ++r) xch[r * T_ + threadIdx.x] = v[r];
+            __syncthreads();
+            const int partner = ((warp ^ (k - 1)) << 5) | (lane ^ 31);
+            if ((warp & (k >> 1)) == 0) {
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], xch[(E - 1 - r) * T_ + partner]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::hi(v[r], xch[(E - 1 - r) * T_ + partner]);
             }
             __syncthreads();
         }
+        // half-cleaners between warps: idx <-> idx ^ (j*1024), j = k/4 .. 1
+#pragma unroll
+        for (int j = k >> 2; j > 0; j >>= 1) {
+#pragma unroll
+            for (int r = 0; r < E; ++r) xch[r * T_ + threadIdx.x] = v[r];
+            __syncthreads();
+            const int partner = ((warp ^ j) << 5) | lane;
+            if ((warp & j) == 0) {
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], xch[r * T_ + partner]);
+            } else {
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::hi(v[r], xch[r * T_ + partner]);
+            }
+            __syncthreads();
+        }
+        warp_half_cleaners<T, E>(v, lane);
     }
 }
 
@@ -263,32 +328,33 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
 }
 
 // ---------------------------------------------------------------------------------------------
-// Sort + accumulate for wide rows (N > 1024): one CTA per row, the row in shared memory.
+// Sort + accumulate for wide rows (1024 < N <= 4096): a CTA of WPR = P/1024 warps per row, keys in
+// registers, running sums in registers, one partial row per CTA.
 // ---------------------------------------------------------------------------------------------
-constexpr int kSortCtaThreads = 512;
-
-__global__ void __launch_bounds__(kSortCtaThreads) k_sort_sum_cta(const float* __restrict__ x, int ldx, int N, int P,
-                                                                   int count, float* __restrict__ partial) {
-    extern __shared__ float srow[];
-    float acc[8];           // P <= 4096 -> at most 8 positions per thread
+template <int WPR>
+__global__ void __launch_bounds__(WPR * 32) k_sort_sum_cta(const float* __restrict__ x, int ldx, int N, int count,
+                                                            float* __restrict__ partial) {
+    __shared__ float xch[WPR * 1024];
+    constexpr int E = 32, T_ = WPR * 32;
+    float acc[E];
 #pragma unroll
-    for (int a = 0; a < 8; ++a) acc[a] = 0.0f;
+    for (int r = 0; r < E; ++r) acc[r] = 0.0f;
     for (int row = blockIdx.x; row < count; row += gridDim.x) {
         const float* src = x + static_cast<size_t>(row) * ldx;
-        for (int e = threadIdx.x; e < P; e += kSortCtaThreads) srow[e] = e < N ? src[e] : INFINITY;
-        __syncthreads();
-        cta_bitonic_sort<float>(srow, P);
+        float v[E];
 #pragma unroll
-        for (int a = 0; a < 8; ++a) {
-            const int e = a * kSortCtaThreads + threadIdx.x;
-            if (e < N) acc[a] += srow[e];
+        for (int r = 0; r < E; ++r) {
+            const int e = r * T_ + threadIdx.x;            // any arrangement sorts; this one loads coalesced
+            v[r] = e < N ? src[e] : INFINITY;
         }
-        __syncthreads();
+        cta_bitonic_sort<float, WPR>(v, xch);
+#pragma unroll
+        for (int r = 0; r < E; ++r) acc[r] += v[r];
     }
 #pragma unroll
-    for (int a = 0; a < 8; ++a) {
-        const int e = a * kSortCtaThreads + threadIdx.x;
-        if (e < N) partial[static_cast<size_t>(blockIdx.x) * N + e] = acc[a];
+    for (int r = 0; r < E; ++r) {
+        const int idx = threadIdx.x * E + r;
+        if (idx < N) partial[static_cast<size_t>(blockIdx.x) * N + idx] = acc[r];
     }
 }
 
@@ -386,20 +452,27 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_debug_sort_warp(const float
     }
 }
 
-__global__ void __launch_bounds__(kSortCtaThreads) k_debug_sort_cta(const float* __restrict__ rows, int n, int P,
-                                                                     int n_rows, float* __restrict__ keys,
-                                                                     int* __restrict__ perm) {
-    extern __shared__ unsigned long long scomp[];
+template <int WPR>
+__global__ void __launch_bounds__(WPR * 32) k_debug_sort_cta(const float* __restrict__ rows, int n, int n_rows,
+                                                              float* __restrict__ keys, int* __restrict__ perm) {
+    __shared__ unsigned long long xch[WPR * 1024];
+    constexpr int E = 32, T_ = WPR * 32;
     for (int row = blockIdx.x; row < n_rows; row += gridDim.x) {
-        for (int e = threadIdx.x; e < P; e += kSortCtaThreads)
-            scomp[e] = e < n ? make_composite(rows[static_cast<size_t>(row) * n + e], e) : ~0ull;
-        __syncthreads();
-        cta_bitonic_sort<unsigned long long>(scomp, P);
-        for (int e = threadIdx.x; e < n; e += kSortCtaThreads) {
-            keys[static_cast<size_t>(row) * n + e] = composite_key(scomp[e]);
-            perm[static_cast<size_t>(row) * n + e] = static_cast<int>(scomp[e] & 0xffffffffu);
+        unsigned long long v[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int e = r * T_ + threadIdx.x;
+            v[r] = e < n ? make_composite(rows[static_cast<size_t>(row) * n + e], e) : ~0ull;
         }
-        __syncthreads();
+        cta_bitonic_sort<unsigned long long, WPR>(v, xch);
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int idx = threadIdx.x * E + r;
+            if (idx < n) {
+                keys[static_cast<size_t>(row) * n + idx] = composite_key(v[r]);
+                perm[static_cast<size_t>(row) * n + idx] = static_cast<int>(v[r] & 0xffffffffu);
+            }
+        }
     }
 }
 
