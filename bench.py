@@ -165,6 +165,8 @@ def main():
     ap.add_argument("--reference-samples", type=int, default=4096)
     ap.add_argument("--cpu-baseline-samples", type=int, default=32768)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-stream", action="store_true")
+    ap.add_argument("--stream-steps", type=int, default=1000)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -282,6 +284,28 @@ def main():
             dist.destroy_process_group()
         return
 
+    # ---- streaming decision latency: push + predict per SGD step inside a CUDA graph -------------------
+    stream_latency = None
+    if not args.no_stream and world == 1:
+        swl = inputs.WORKLOADS["stream"]
+        sweights = inputs.workload_weights(swl)
+        strace = inputs.workload_trace(swl, swl.window + 8 + args.stream_steps)
+        sctx = binding.Cutoff(swl.N, swl.D, swl.H, swl.lag, swl.S, precision=swl.precision, seed=7, device=local_rank,
+                              stream=stream.cuda_stream, flags=binding.FLAG_GRAPH)
+        sctx.load_weights(sweights)
+        for x in strace[: swl.window + 8]:
+            sctx.step(x)
+        lat = []
+        for x in strace[swl.window + 8:]:
+            t0 = time.perf_counter()
+            sctx.step(x)
+            lat.append((time.perf_counter() - t0) * 1e6)
+        lat.sort()
+        stream_latency = {"workload": "stream", "N": swl.N, "S": swl.S, "steps": len(lat),
+                          "p50_us": lat[len(lat) // 2], "p99_us": lat[int(len(lat) * 0.99)],
+                          "how": "host clock around cutoff_step (host run-times in, cutoff out), CUDA graph replay"}
+        sctx.close()
+
     # ---- roofline of the dominant stage -----------------------------------------------------------
     peaks = {}
     try:
@@ -325,6 +349,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
                 "h2d_bytes_per_step": 4 * wl.N, "d2h_bytes_per_step": 40 + 8 * wl.N},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline,
+        "stream_latency": stream_latency,
         "timed_region_wall_s": round(wall, 3),
     }
     print(json.dumps(line))

@@ -86,7 +86,9 @@ typedef struct {
     int64_t sample_offset;      /* index of this context's first sample in the global draw         */
     int64_t total_samples;      /* samples of the whole decision (0 means n_samples); used only to
                                    normalise when several contexts share one decision              */
-    void*   stream;             /* cudaStream_t the kernels run on; NULL = the default stream      */
+    void*   stream;             /* cudaStream_t the kernels run on; NULL = the default stream (with
+                                   CUTOFF_FLAG_GRAPH: a stream the context creates, because the
+                                   default stream cannot be captured)                              */
     uint64_t seed;              /* Philox key                                                      */
 } cutoff_config;
 
@@ -130,6 +132,15 @@ int cutoff_predict(cutoff_ctx* ctx, int32_t* c_out);
  * and read the result.  cutoff_fetch returns what cutoff_predict would have returned. */
 int cutoff_predict_async(cutoff_ctx* ctx);
 int cutoff_fetch(cutoff_ctx* ctx, int32_t* c_out);
+
+/* One iteration of the parameter server's loop in a single call: append this step's run-times
+ * (host, N floats, as for cutoff_push) and return the cutoff for the next step (as cutoff_predict).
+ * With CUTOFF_FLAG_GRAPH the copy, the push and all kernels of the decision are captured into a
+ * CUDA graph the first time the window is full and a decision has already run; later calls
+ * replay it (no argument changes between replays: window position, normaliser and decision
+ * counter live in device memory).  Without the flag it is cutoff_push followed by cutoff_predict.
+ * Returns what cutoff_predict returns.  Errors: BAD_ARG, BAD_VALUE, STATE, CUDA, TIMEOUT. */
+int cutoff_step(cutoff_ctx* ctx, const float* runtimes_sec, int32_t* c_out);
 
 /* Results of the last completed decision.  Either pointer may be NULL.
  * exp_order_stats_sec (host, N floats): E[x~_(j)] in seconds, ascending.

@@ -26,7 +26,7 @@ BLOB_MAGIC = 0x31465443
 
 EXPORTS = (
     "cutoff_create", "cutoff_destroy", "cutoff_load_weights", "cutoff_push", "cutoff_push_async",
-    "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_get_stats",
+    "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_step", "cutoff_get_stats",
     "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
@@ -71,6 +71,7 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_predict": (C.c_int, [vp, i32p]),
         "cutoff_predict_async": (C.c_int, [vp]),
         "cutoff_fetch": (C.c_int, [vp, i32p]),
+        "cutoff_step": (C.c_int, [vp, vp, i32p]),
         "cutoff_get_stats": (C.c_int, [vp, vp, vp]),
         "cutoff_get_partial_sums": (C.c_int, [vp, vp]),
         "cutoff_decide_from_sums": (C.c_int, [vp, vp, i32p]),
@@ -184,6 +185,15 @@ class Cutoff:
     def fetch(self):
         c = C.c_int32(0)
         rc = self._check(self._lib.cutoff_fetch(self._h, C.byref(c)), "cutoff_fetch")
+        return rc, c.value
+
+    def step(self, runtimes_sec: np.ndarray):
+        """push + predict in one call (a CUDA-graph replay when the context has FLAG_GRAPH); returns (code, c)."""
+        a = np.ascontiguousarray(runtimes_sec, dtype=np.float32)
+        if a.shape != (self.N,):
+            raise ValueError("expected N run-times")
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_step(self._h, a.ctypes.data, C.byref(c)), "cutoff_step")
         return rc, c.value
 
     def get_stats(self):

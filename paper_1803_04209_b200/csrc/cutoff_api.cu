@@ -38,6 +38,7 @@ struct cutoff_ctx {
     int n_chunks = 0;
     int sort_grid = 0;      // CTAs of the sort kernel per chunk (= partial rows per chunk)
     cudaStream_t stream = nullptr;
+    bool owns_stream = false;       // the context created `stream` itself (graph mode with a NULL stream)
 
     float* d_blob = nullptr;        // tensors as loaded
     float* d_WT = nullptr;          // transposed copies WzT, W1T, W3T: 3 x [D][H]
@@ -73,6 +74,11 @@ struct cutoff_ctx {
     bool ev_created = false;
     float stage_ms[kNumStages]{};
     int timed_chunks = 0;
+
+    cudaGraph_t graph = nullptr;            // captured push + decision (CUTOFF_FLAG_GRAPH)
+    cudaGraphExec_t graph_exec = nullptr;
+    int graph_kernels = 0;                  // kernels one replay launches
+    bool decided_once = false;              // a decision has run outside capture (function attributes are set)
 
     int64_t launches = 0;
     std::string last_error;
@@ -111,6 +117,9 @@ void free_all(cutoff_ctx* c) {
     cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->h_state) cudaFreeHost(c->h_state);
+    if (c->owns_stream && c->stream) cudaStreamDestroy(c->stream);
+    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    if (c->graph) cudaGraphDestroy(c->graph);
     if (c->ev_created)
         for (auto& row : c->ev)
             for (auto& e : row)
@@ -179,8 +188,8 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
     if (resident <= 200 * 1024) {
         // all weights fit: one persistent CTA per SM, as many as there are warp batches to hand out
         const int batch = 32 / ChainShape<D>::G * ChainShape<D>::SPL;
-        const int ctas_needed = ceil_div(ceil_div(count, batch), kChainResidentThreads / 32);
-        const int grid = ctas_needed < c->sm_count ? ctas_needed : c->sm_count;
+        const int batches = ceil_div(count, batch);
+        const int grid = batches < c->sm_count ? batches : c->sm_count;
         k_chain_resident<D><<<grid, kChainResidentThreads, resident, c->stream>>>(c->m, c->d_hlr, c->d_state, key,
                                                                                 sample_base, count, round_v, c->d_v);
     } else {
@@ -377,6 +386,11 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     } while (0)
 
     CREATE_CHECK(cudaSetDevice(cfg->device));
+    if ((cfg->flags & CUTOFF_FLAG_GRAPH) && !c->stream) {
+        // the default stream cannot be captured: graph mode without a caller stream runs on its own
+        CREATE_CHECK(cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking));
+        c->owns_stream = true;
+    }
     cudaDeviceProp prop;
     CREATE_CHECK(cudaGetDeviceProperties(&prop, cfg->device));
     c->sm_count = prop.multiProcessorCount;
@@ -568,6 +582,7 @@ int cutoff_fetch(cutoff_ctx* c, int32_t* c_out) {
     const int rc = collect_timing(c);
     if (rc) return rc;
     c->have_result = true;
+    c->decided_once = true;
     *c_out = c->h_state->c_star;
     return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
 }
@@ -577,6 +592,63 @@ int cutoff_predict(cutoff_ctx* c, int32_t* c_out) {
     const int rc = cutoff_predict_async(c);
     if (rc < 0) return rc;
     return cutoff_fetch(c, c_out);
+}
+
+// Capture "land the staged run-times, push, decide, read back the state" once; replays need no
+// changing argument because the window position, the normaliser and the decision counter live
+// in device memory.
+static int build_graph(cutoff_ctx* c) {
+    const int64_t launches_before = c->launches;
+    CU_CHECK(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+    cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, cudaMemcpyHostToDevice, c->stream);
+    k_push<<<1, kPushThreads, 0, c->stream>>>(c->d_stage, c->d_ring, c->d_state, c->N, c->W);
+    c->launches += 1;
+    const bool timing = c->timing;
+    c->timing = false;
+    const int rc = enqueue_decision(c);
+    c->timing = timing;
+    cudaGraph_t g = nullptr;
+    const cudaError_t end = cudaStreamEndCapture(c->stream, &g);
+    c->graph_kernels = static_cast<int>(c->launches - launches_before);
+    c->launches = launches_before;                 // nothing ran yet
+    if (rc != CUTOFF_OK || end != cudaSuccess || !g) {
+        if (g) cudaGraphDestroy(g);
+        c->last_error = std::string("graph capture failed: ") + cudaGetErrorString(end);
+        cudaGetLastError();
+        return CUTOFF_ERR_CUDA;
+    }
+    c->graph = g;
+    CU_CHECK(c, cudaGraphInstantiate(&c->graph_exec, c->graph, 0));
+    return CUTOFF_OK;
+}
+
+int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
+    if (!c || !runtimes_sec || !c_out) return CUTOFF_ERR_BAD_ARG;
+    if (!c->weights_loaded || c->pending) return CUTOFF_ERR_STATE;
+    const bool replay = (c->cfg.flags & CUTOFF_FLAG_GRAPH) && c->decided_once &&
+                        c->pushes + 1 >= static_cast<uint32_t>(c->W);
+    if (!replay) {
+        const int rc = cutoff_push(c, runtimes_sec, 0, nullptr);
+        if (rc < 0) return rc;
+        return cutoff_predict(c, c_out);
+    }
+    for (int j = 0; j < c->N; ++j)
+        if (!(runtimes_sec[j] > 0.0f) || !std::isfinite(runtimes_sec[j])) return CUTOFF_ERR_BAD_VALUE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (!c->graph_exec) {
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));
+        const int rc = build_graph(c);
+        if (rc) return rc;
+    }
+    std::memcpy(c->h_stage, runtimes_sec, sizeof(float) * c->N);     // the stream is idle: every call ends synchronised
+    CU_CHECK(c, cudaGraphLaunch(c->graph_exec, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    c->launches += c->graph_kernels;
+    c->pushes += 1;
+    if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
+    c->have_result = true;
+    *c_out = c->h_state->c_star;
+    return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
 }
 
 int cutoff_get_stats(cutoff_ctx* c, float* e_out, float* omega_out) {

@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float
 
 // Variant 2: every weight of the chain resident in shared memory, one persistent CTA per SM.
 // The weights are staged once; after that the warps never synchronise: warp w of the grid takes
-// the sample batches w, w + (warps in the grid), ... (a batch = the samples one warp covers).
+// the sample batches blockIdx + gridDim * w, + (warps in the grid), ... (a batch = the samples one warp covers).
 constexpr int kChainResidentThreads = 512;
 
 inline size_t chain_resident_smem_floats(int D, int H, int W) {
@@ -467,7 +467,8 @@ k_chain_resident(ModelDev m, const float* __restrict__ hlr, const DevState* __re
     const int warps_in_grid = gridDim.x * (kChainResidentThreads / 32);
     const int n_batches = ceil_div(count, kBatch);
     const uint32_t step = st->step;
-    for (int b = blockIdx.x * (kChainResidentThreads / 32) + (threadIdx.x >> 5); b < n_batches; b += warps_in_grid) {
+    // consecutive batches go to different CTAs, so that a small decision still spreads over all SMs
+    for (int b = blockIdx.x + gridDim.x * (threadIdx.x >> 5); b < n_batches; b += warps_in_grid) {
         const int k0 = b * kBatch + (lane / G) * SPL;
         const ChainNoise nz{key, step, sample_base + static_cast<uint32_t>(k0)};
         float z[SPL][D];

@@ -174,6 +174,37 @@ def test_streaming_loop_matches_oracle():
         orc.push(x)
 
 
+def test_graph_replay_equals_plain_calls_and_oracle():
+    # the streaming loop: step() = push + predict; with the graph flag the same kernels are replayed
+    wl = inputs.WORKLOADS["stream"]
+    S = 512
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, wl.window + 12)
+    plain = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED)
+    graph = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED, flags=binding.FLAG_GRAPH)
+    orc = O.CutoffOracle(w, wl.lag, S, seed=SEED)
+    plain.load_weights(w)
+    graph.load_weights(w)
+    launches = []
+    for t, x in enumerate(trace):
+        orc.push(x)
+        code_o, c_o, e_o, om_o = orc.predict()
+        rp = plain.step(x)
+        rg = graph.step(x)
+        assert rp == rg and rp[0] == code_o
+        launches.append(graph.launch_count())
+        if code_o == O.OK:
+            e_p, e_g = plain.get_stats()[0], graph.get_stats()[0]
+            assert np.array_equal(e_p, e_g)                     # same kernels, same bits
+            assert np.max(np.abs(e_g - e_o) / e_o[-1]) <= TOL_E
+            top = np.sort(om_o[np.isfinite(om_o)])[-2:]
+            assert rg[1] == c_o or (top[1] - top[0]) <= TOL_E * top[1]
+    assert launches[-1] - launches[-2] == launches[-2] - launches[-3] > 0    # replays are counted
+    with pytest.raises(binding.CutoffError) as e:
+        graph.step(np.zeros(wl.N, dtype=np.float32))
+    assert e.value.code == binding.ERR_BAD_VALUE
+
+
 def test_device_pushes_equal_host_pushes():
     import torch
     wl = inputs.WORKLOADS["n128"]
