@@ -16,7 +16,7 @@ struct DevState {
     int32_t error_flags;    // bit 0: a pushed value was not finite or not > 0; bit 1: device wait timed out
     int32_t c_star;         // last decision
     int32_t code;           // 0 ok, 2 degenerate
-    int32_t pad;
+    uint32_t ticket;        // CTAs that have finished their column sums (self-resetting)
 };
 
 constexpr int kErrBadValue = 1;

@@ -264,10 +264,29 @@ void launch_emission(cutoff_ctx* c, uint32_t sample_base, int count) {
     c->launches += 1;
 }
 
+template <int HQ>
+void launch_rnn_resident(cutoff_ctx* c) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_enc_rnn_resident<HQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        attr_set = true;
+    }
+    const size_t smem = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float);
+    k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_proj, c->d_hlr);
+}
+
 void launch_encoder(cutoff_ctx* c) {
     dim3 grid(ceil_div(c->H, kProjWarps), 2);
     k_enc_proj<<<grid, kProjWarps * 32, 0, c->stream>>>(c->m, c->d_ring, c->d_state, c->d_proj);
-    k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_hlr);
+    const bool fits = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float) <= 200 * 1024;
+    switch (fits ? c->H : 0) {
+        case 32: launch_rnn_resident<8>(c); break;
+        case 64: launch_rnn_resident<16>(c); break;
+        case 128: launch_rnn_resident<32>(c); break;
+        case 256: launch_rnn_resident<64>(c); break;
+        default:
+            k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_hlr);
+    }
     c->launches += 2;
 }
 
@@ -302,11 +321,11 @@ int enqueue_decision(cutoff_ctx* c) {
         if (rc) return rc;
         if (timed) cudaEventRecord(c->ev[4][ch], c->stream);
     }
-    k_colsum<<<ceil_div(c->N, 256), 256, 0, c->stream>>>(c->d_partial, c->n_chunks * c->sort_grid, c->N, c->d_sums);
     const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
-    k_decide<<<1, kDecideThreads, 0, c->stream>>>(c->d_sums, c->N, 1.0 / static_cast<double>(total), c->d_state, 1,
-                                                  c->d_E, c->d_omega);
-    c->launches += 2;
+    k_colsum_decide<<<ceil_div(c->N, 32), kColsumThreads, 0, c->stream>>>(c->d_partial, c->n_chunks * c->sort_grid, c->N,
+                                                                         c->d_sums, 1.0 / static_cast<double>(total),
+                                                                         c->d_state, c->d_E, c->d_omega);
+    c->launches += 1;
     if (timed) cudaEventRecord(c->ev[5][0], c->stream);
     c->timed_chunks = timed ? c->n_chunks : 0;
     CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));

@@ -80,10 +80,26 @@ __global__ void __launch_bounds__(kProjWarps * 32) k_enc_proj(ModelDev m, const 
             const int t = min(t0 + tt, m.W - 1);
             row[tt] = ring + static_cast<size_t>((pushes + t) % m.W) * m.N;
         }
-        for (int j = lane; j < m.N; j += 32) {
-            const float w = Wx[j];
+        if ((m.N & 3) == 0) {
+            // 16-byte loads, four independent iterations in flight
+#pragma unroll 4
+            for (int j = 4 * lane; j < m.N; j += 128) {
+                const float4 w = *reinterpret_cast<const float4*>(Wx + j);
 #pragma unroll
-            for (int tt = 0; tt < kProjChunk; ++tt) acc[tt] = fmaf(w, row[tt][j] * inv_scale, acc[tt]);
+                for (int tt = 0; tt < kProjChunk; ++tt) {
+                    const float4 xv = *reinterpret_cast<const float4*>(row[tt] + j);
+                    acc[tt] = fmaf(w.x, xv.x * inv_scale, acc[tt]);
+                    acc[tt] = fmaf(w.y, xv.y * inv_scale, acc[tt]);
+                    acc[tt] = fmaf(w.z, xv.z * inv_scale, acc[tt]);
+                    acc[tt] = fmaf(w.w, xv.w * inv_scale, acc[tt]);
+                }
+            }
+        } else {
+            for (int j = lane; j < m.N; j += 32) {
+                const float w = Wx[j];
+#pragma unroll
+                for (int tt = 0; tt < kProjChunk; ++tt) acc[tt] = fmaf(w, row[tt][j] * inv_scale, acc[tt]);
+            }
         }
 #pragma unroll
         for (int tt = 0; tt < kProjChunk; ++tt) {
@@ -133,6 +149,73 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
         }
         __syncthreads();
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Encoder, part 2, latency version for H <= 256: the recurrence matrix never leaves the SM.
+// One CTA per direction, 4 threads per hidden unit; thread (i, q) owns columns q*H/4 .. of row i:
+// the first 32 of them in registers, the rest (H = 256 only) in shared memory, laid out
+// [column group][thread] so that a warp's 16-byte reads are contiguous.  The state is
+// double-buffered in shared memory, so a step costs one __syncthreads.
+// ---------------------------------------------------------------------------------------------
+template <int HQ>   // HQ = H / 4
+__global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const float* __restrict__ proj,
+                                                              float* __restrict__ hlr /*[2][W][H]*/) {
+    constexpr int H = 4 * HQ, T = 16 * HQ, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ, PAD = HQ + 4;
+    extern __shared__ __align__(16) float sm_rr[];
+    float* state = sm_rr;                         // [2][4][PAD]
+    float* sproj = state + 2 * 4 * PAD;           // [W][H]
+    float* swh = sproj + m.W * H;                 // [SQ/4][T][4]
+    const int dir = blockIdx.x;
+    const int t = threadIdx.x, i = t >> 2, q = t & 3;
+    const float* Wh = (dir ? m.Whb : m.Whf) + static_cast<size_t>(i) * H + q * HQ;
+    const float* init = dir ? m.b0 : m.a0;
+    float w[RQ];
+#pragma unroll
+    for (int j4 = 0; j4 < RQ / 4; ++j4) {
+        const float4 v = *reinterpret_cast<const float4*>(Wh + 4 * j4);
+        w[4 * j4 + 0] = v.x; w[4 * j4 + 1] = v.y; w[4 * j4 + 2] = v.z; w[4 * j4 + 3] = v.w;
+    }
+#pragma unroll
+    for (int j4 = 0; j4 < SQ / 4; ++j4)
+        *reinterpret_cast<float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4) =
+            *reinterpret_cast<const float4*>(Wh + RQ + 4 * j4);
+    for (int idx = t; idx < m.W * H; idx += T) sproj[idx] = proj[static_cast<size_t>(dir) * m.W * H + idx];
+    if (t < H) state[(t / HQ) * PAD + (t % HQ)] = init[t];
+    __syncthreads();
+    int cur = 0;
+    for (int s = 0; s < m.W; ++s) {
+        const int tt = dir ? (m.W - 1 - s) : s;
+        const float* st = state + cur * 4 * PAD + q * PAD;
+        float acc = 0.0f;
+#pragma unroll
+        for (int j4 = 0; j4 < RQ / 4; ++j4) {
+            const float4 v = *reinterpret_cast<const float4*>(st + 4 * j4);
+            acc = fmaf(w[4 * j4 + 0], v.x, acc); acc = fmaf(w[4 * j4 + 1], v.y, acc);
+            acc = fmaf(w[4 * j4 + 2], v.z, acc); acc = fmaf(w[4 * j4 + 3], v.w, acc);
+        }
+#pragma unroll
+        for (int j4 = 0; j4 < SQ / 4; ++j4) {
+            const float4 v = *reinterpret_cast<const float4*>(st + RQ + 4 * j4);
+            const float4 ww = *reinterpret_cast<const float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4);
+            acc = fmaf(ww.x, v.x, acc); acc = fmaf(ww.y, v.y, acc);
+            acc = fmaf(ww.z, v.z, acc); acc = fmaf(ww.w, v.w, acc);
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        if (q == 0) {
+            const float v = fmaxf(acc + sproj[tt * H + i], 0.0f);
+            state[(cur ^ 1) * 4 * PAD + (i / HQ) * PAD + (i % HQ)] = v;
+            hlr[(static_cast<size_t>(dir) * m.W + tt) * H + i] = v;
+        }
+        __syncthreads();
+        cur ^= 1;
+    }
+}
+
+inline size_t enc_rnn_resident_smem_floats(int H, int W) {
+    const int HQ = H / 4, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ;
+    return 2 * 4 * (HQ + 4) + static_cast<size_t>(W) * H + static_cast<size_t>(SQ) * 4 * H;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -359,33 +359,19 @@ __global__ void __launch_bounds__(WPR * 32) k_sort_sum_cta(const float* __restri
 }
 
 // ---------------------------------------------------------------------------------------------
-// Column sums of the partial rows, in a fixed order, in double.
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_colsum(const float* __restrict__ partial, int n_part, int N,
-                                                double* __restrict__ sums) {
-    const int j = blockIdx.x * 256 + threadIdx.x;
-    if (j >= N) return;
-    double s = 0.0;
-    for (int p = 0; p < n_part; ++p) s += static_cast<double>(partial[static_cast<size_t>(p) * N + j]);
-    sums[j] = s;
-}
-
-// ---------------------------------------------------------------------------------------------
 // Decision: E_j = s * sums_j / S (seconds), Omega(c) = c / E_c (minus infinity where E_c <= 0),
 // c* = the largest c attaining the maximum; c* = N and code 2 if no c is admissible.
-// One CTA.  Advances the decision counter when asked to.
+// Executed by one whole CTA of THREADS threads.  Advances the decision counter when asked to.
 // ---------------------------------------------------------------------------------------------
-constexpr int kDecideThreads = 1024;
-
-__global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restrict__ sums, int N, double inv_samples,
-                                                            DevState* st, int advance, float* __restrict__ e_out,
-                                                            float* __restrict__ omega_out) {
-    __shared__ double best_val[kDecideThreads / 32];
-    __shared__ int best_idx[kDecideThreads / 32];
+template <int THREADS>
+__device__ __forceinline__ void decide_block(const double* sums, int N, double inv_samples, DevState* st, int advance,
+                                             float* __restrict__ e_out, float* __restrict__ omega_out) {
+    __shared__ double best_val[THREADS / 32];
+    __shared__ int best_idx[THREADS / 32];
     const double scale = static_cast<double>(st->scale);
     double bv = -INFINITY;
     int bi = 0;                                   // 0 = nothing admissible yet
-    for (int j = threadIdx.x; j < N; j += kDecideThreads) {
+    for (int j = threadIdx.x; j < N; j += THREADS) {
         const double e = scale * sums[j] * inv_samples;
         const double om = e > 0.0 ? static_cast<double>(j + 1) / e : -INFINITY;
         e_out[j] = static_cast<float>(e);
@@ -402,7 +388,7 @@ __global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restr
     if (lane == 0) { best_val[warp] = bv; best_idx[warp] = bi; }
     __syncthreads();
     if (threadIdx.x == 0) {
-        for (int w = 1; w < kDecideThreads / 32; ++w) {
+        for (int w = 1; w < THREADS / 32; ++w) {
             const double ov = best_val[w];
             const int oi = best_idx[w];
             if (oi != 0 && (bi == 0 || ov > bv || (ov == bv && oi > bi))) { bv = ov; bi = oi; }
@@ -411,6 +397,75 @@ __global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restr
         st->code = bi == 0 ? 2 : 0;
         if (advance) st->step += 1;
     }
+}
+
+constexpr int kDecideThreads = 1024;
+
+__global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restrict__ sums, int N, double inv_samples,
+                                                            DevState* st, int advance, float* __restrict__ e_out,
+                                                            float* __restrict__ omega_out) {
+    decide_block<kDecideThreads>(sums, N, inv_samples, st, advance, e_out, omega_out);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Column sums of the partial rows, in a fixed order, in double, followed by the decision in the
+// CTA that finishes last (a ticket counter in the device state; nobody waits on anybody).
+// A CTA covers 32 columns with 8 row slices; slice s adds rows s, s+8, ...; the slices are then
+// added in order.
+// ---------------------------------------------------------------------------------------------
+constexpr int kColsumThreads = 256;
+
+__global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* __restrict__ partial, int n_part, int N,
+                                                                   double* sums, double inv_samples, DevState* st,
+                                                                   float* __restrict__ e_out, float* __restrict__ omega_out) {
+    __shared__ double red[8][32];
+    __shared__ bool is_last;
+    const int col = blockIdx.x * 32 + (threadIdx.x & 31), slice = threadIdx.x >> 5;
+    double s = 0.0;
+    if (col < N) {
+        int p = slice;
+        for (; p + 24 < n_part; p += 32) {
+            const float a = partial[static_cast<size_t>(p) * N + col];
+            const float b = partial[static_cast<size_t>(p + 8) * N + col];
+            const float c = partial[static_cast<size_t>(p + 16) * N + col];
+            const float d = partial[static_cast<size_t>(p + 24) * N + col];
+            s += static_cast<double>(a);
+            s += static_cast<double>(b);
+            s += static_cast<double>(c);
+            s += static_cast<double>(d);
+        }
+        for (; p < n_part; p += 8) s += static_cast<double>(partial[static_cast<size_t>(p) * N + col]);
+    }
+    red[slice][threadIdx.x & 31] = s;
+    __syncthreads();
+    if (slice == 0 && col < N) {
+        double total = 0.0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) total += red[k][threadIdx.x];
+        sums[col] = total;
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t ticket = atomicAdd(&st->ticket, 1u);
+        is_last = ticket == gridDim.x - 1;
+        if (is_last) st->ticket = 0;
+    }
+    __syncthreads();
+    if (is_last) {
+        __threadfence();
+        decide_block<kColsumThreads>(sums, N, inv_samples, st, 1, e_out, omega_out);
+    }
+}
+
+// Plain column sums of partial rows (fixed order, double): one thread per column.
+__global__ void __launch_bounds__(256) k_colsum(const float* __restrict__ partial, int n_part, int N,
+                                                double* __restrict__ sums) {
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= N) return;
+    double s = 0.0;
+    for (int p = 0; p < n_part; ++p) s += static_cast<double>(partial[static_cast<size_t>(p) * N + j]);
+    sums[j] = s;
 }
 
 // ---------------------------------------------------------------------------------------------
