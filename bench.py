@@ -185,7 +185,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_1803_04209_b200 import binding, build
+    from paper_1803_04209_b200 import binding, build, sharding
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -198,8 +198,11 @@ def main():
     stream = torch.cuda.current_stream()
 
     # N ranks share one decision: each draws S samples with global sample indices (weak scaling)
-    ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, wl.S, precision=wl.precision, seed=2024, device=local_rank,
-                         stream=stream.cuda_stream, sample_offset=rank * wl.S, total_samples=world * wl.S)
+    shard = sharding.shard_config(rank, world, wl.S)
+    ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, shard["n_samples"], precision=wl.precision, seed=2024,
+                         device=local_rank, stream=stream.cuda_stream, sample_offset=shard["sample_offset"],
+                         total_samples=shard["total_samples"])
+    shared = sharding.ShardedDecision(ctx, device="cuda") if world > 1 else None
     ctx.load_weights(weights)
     if args.pass_rows:
         ctx.set_option("pass_rows", args.pass_rows)
@@ -208,16 +211,14 @@ def main():
         ctx.push(x)
     dev_trace = torch.from_numpy(trace[n_hist:]).cuda()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-    sums_dev = torch.empty(wl.N, dtype=torch.float64, device="cuda")
 
     def step_device(i):
         ctx.push_async(dev_trace[i])
-        ctx.predict_async()
-        code, c = ctx.fetch()
         if world > 1:
-            sums_dev.copy_(torch.from_numpy(ctx.get_partial_sums()))
-            dist.all_reduce(sums_dev)
-            code, c = ctx.decide_from_sums(sums_dev.cpu().numpy())
+            code, c = shared.predict()         # local samples, one all-reduce of N sums, shared decision
+        else:
+            ctx.predict_async()
+            code, c = ctx.fetch()
         return c
 
     def barrier():
@@ -265,11 +266,7 @@ def main():
     t0 = time.perf_counter()
     for i in range(args.steps):
         ctx.push(host_trace[args.warmup + i])
-        code, c = ctx.predict()
-        if world > 1:
-            sums_dev.copy_(torch.from_numpy(ctx.get_partial_sums()))
-            dist.all_reduce(sums_dev)
-            code, c = ctx.decide_from_sums(sums_dev.cpu().numpy())
+        code, c = shared.predict() if world > 1 else ctx.predict()
         e_sec, omega = ctx.get_stats()
     barrier()
     e2e_sec = (time.perf_counter() - t0) / args.steps

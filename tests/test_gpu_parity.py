@@ -153,6 +153,35 @@ def test_decision_tensor_cores(name, S, offsets):
     assert_decision_close(gpu, orc.predict(), wl.N)
 
 
+@pytest.mark.parametrize("name", ["n1024", "n4096"])
+def test_full_size_sampled_rows_and_invariants(name):
+    # the workload at its full size, in the launch configuration bench.py times
+    wl, gpu, orc, prec = make_pair(name, steps=inputs.WORKLOADS[name].window + 7)
+    S = wl.S
+    for k0 in (0, S // 2 - 17, S - 48):                    # rows the oracle computes one by one
+        x_gpu = gpu.debug_samples(k0, 48)
+        x_orc = orc.samples(np.arange(k0, k0 + 48))
+        assert_samples_close(x_gpu, x_orc, TOL_X[prec])
+    x_all = gpu.debug_samples(0, S).astype(np.float64)     # properties that hold at any size
+    code, c = gpu.predict()
+    e, om = gpu.get_stats()
+    sums = gpu.get_partial_sums()
+    s_norm = orc.scale()
+    assert code == binding.OK
+    assert np.all(np.diff(e) >= 0)                                                    # order statistics ascend
+    assert abs(sums.sum() - x_all.sum()) <= 1e-6 * np.abs(x_all).sum()                # sorting permutes each row
+    assert x_all.min() * s_norm <= e[0] * (1 + 1e-6) and e[-1] <= x_all.max() * s_norm * (1 + 1e-6)
+    want = s_norm * np.sort(x_all, axis=1).mean(axis=0)                               # numpy sort of the GPU's own draws
+    assert np.max(np.abs(e - want) / want[-1]) <= 1e-6
+    finite = np.isfinite(om)
+    assert c == int(np.flatnonzero(om == om[finite].max()).max()) + 1                 # largest c attaining the maximum
+
+
+def test_full_size_decision_against_the_full_oracle():
+    wl, gpu, orc, prec = make_pair("n1024", steps=inputs.WORKLOADS["n1024"].window + 7)
+    assert_decision_close(gpu, orc.predict(), wl.N)
+
+
 def test_streaming_loop_matches_oracle():
     wl = inputs.WORKLOADS["tiny"]
     w = inputs.workload_weights(wl)
