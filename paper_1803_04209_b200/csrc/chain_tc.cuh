@@ -1,0 +1,352 @@
+// Per-sample chain (guide steps, transition, emission hidden layer) on the tcgen05 tensor cores,
+// for latent size 16 and hidden width 64..256, operands in tf32.
+//
+// A CTA walks over tiles of 128 samples; sample r of the tile is TMEM lane r.  Every layer pair
+//      hidden = act(A z + a)          (M=128, N=H, K=16)
+//      out    = B hidden (+ b)        (M=128, N=16 or 32, K=H)
+// is two UMMA groups.  The first writes the hidden pre-activations to TMEM columns [0, H); the
+// epilogue warps read them 64 hidden units ("chunk") at a time, apply bias and activation, round
+// to tf32 and store the chunk as a K-major, 128-byte-swizzled A operand in one of two shared
+// memory buffers; the MMA warp multiplies chunk c with the matching K blocks of B while the
+// epilogue produces chunk c+1.  The second result (mu, or mean | logvar) is read back by all
+// epilogue warps, which draw the noise, form the next latent and store it as the next A operand.
+// The last layer's hidden vector v goes to global memory for the emission output GEMM.
+//
+// All weight operands live in shared memory for the whole kernel: the host prepares their
+// swizzled image once, the CTA copies it in at start.  Latent rows are 128 bytes wide (32 tf32)
+// although K = 16: Wz and W1 share one tile (columns 0..15 and 16..31), so the MMA for the
+// transition simply starts 64 bytes into the rows.
+//
+// Warp 0 issues the MMAs and owns TMEM; warps 1..16 are the epilogue: warp w serves TMEM lanes
+// 32*(w%4).. and column group cg = (w-1)/4: 16 of each chunk's 64 columns and the latent
+// dimensions 4cg..4cg+3 (one Philox call per stream and sample, as everywhere else).
+// Every mbarrier wait is bounded (see async.cuh).
+#pragma once
+#include "emit_tc.cuh"
+
+namespace cutoff {
+namespace tc {
+
+constexpr int kChainEpiWarps = 16;
+constexpr int kChainTcThreads = (1 + kChainEpiWarps) * 32;
+constexpr int kChainD = 16;
+constexpr int kColMu = 256, kColHead = 320;      // TMEM columns of the second-GEMM results
+
+struct ChainTcArgs {
+    const float* image;         // swizzled operand tiles: [Wz|W1] (H x 32), W3 (H x 32), Wmu (H/32 x 16 x 32), W2 (H/32 x 32 x 32)
+    const float *bz, *b1, *b3, *bmu, *bsig, *Wsig, *b2, *z0;
+    const float* hlr;           // [2][W][H] h_left, h_right
+    DevState* st;
+    NoiseKey key;
+    uint32_t sample_base;
+    int count, H, W, round_v;
+    float* v_out;               // [count][H]
+};
+
+inline size_t chain_tc_image_floats(int H) { return static_cast<size_t>(H) * (32 + 32 + 16 + 32); }
+
+inline size_t chain_tc_smem_bytes(int H, int W) {
+    const size_t tiles = chain_tc_image_floats(H) * 4 + 128 * 128 + 2 * 2 * 128 * 128;
+    const size_t floats = 3 * static_cast<size_t>(H) + static_cast<size_t>(W) * H + 16 * 16 + 16 + 16 + 32 + 16;
+    return 1024 + tiles + floats * 4 + 256;
+}
+
+// byte offset of the 16-byte chunk `chunk` of row `row` in a K-major tile with 128-byte swizzled rows
+__device__ __forceinline__ uint32_t sw128(int row, int chunk) {
+    return static_cast<uint32_t>((row >> 3) * 1024 + (row & 7) * 128 + ((chunk ^ (row & 7)) << 4));
+}
+
+__device__ __forceinline__ uint32_t instr_desc_tf32(int n) {      // D = f32, A = B = tf32, K-major, M = 128
+    return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+__device__ __forceinline__ float tf32_rna(float x) {
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, float c, float d) {
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+
+__device__ __forceinline__ float softplus_fast(float x) {          // ln(1 + e^x)
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * 1.4426950408889634f));
+    return x > 15.0f ? x : 0.6931471805599453f * __log2f(1.0f + e);
+}
+
+__global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const int H = a.H, W = a.W;
+    const int n_chunks = H / 64, kblocks = H / 32;
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* gen = smem_raw + (base - raw);
+    // operand tiles
+    const uint32_t t_zw1 = base;
+    const uint32_t t_w3 = t_zw1 + H * 128;
+    const uint32_t t_wmu = t_w3 + H * 128;
+    const uint32_t t_w2 = t_wmu + H * 64;
+    const uint32_t t_z = t_w2 + H * 128;
+    const uint32_t t_hb = t_z + 128 * 128;                       // two buffers of 32 KB
+    const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u;
+    // fp32 side tables
+    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 128 * 128 + 2 * 32768);    // bz * 2 log2(e)
+    float* sb1 = sbzs + H;
+    float* sb3 = sb1 + H;
+    float* slr = sb3 + H;                    // [W][H]  (h_left + h_right + 1) / 3
+    float* sWsig = slr + W * H;              // [16][16]
+    float* sbmu = sWsig + 256;
+    float* sbsig = sbmu + 16;
+    float* sb2 = sbsig + 16;                 // [32]
+    float* sz0 = sb2 + 32;                   // [16]
+    const uint32_t bars = smem_u32(sz0 + 16);
+    const uint32_t bar_z = bars, bar_p = bars + 8, bar_h = bars + 16 /*2*/, bar_hfree = bars + 32 /*2*/,
+                   bar_acc2 = bars + 48, bar_drain = bars + 56;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sz0 + 16 + 16);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sz0 + 16 + 18);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- one-time set-up: operand image, side tables, barriers, TMEM --------------------------------
+    {
+        const float4* src = reinterpret_cast<const float4*>(a.image);
+        float4* dst = reinterpret_cast<float4*>(gen);
+        for (uint32_t i = threadIdx.x; i < image_bytes / 16; i += kChainTcThreads) dst[i] = src[i];
+        for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
+            sbzs[i] = a.bz[i] * 2.8853900817779268f;
+            sb1[i] = a.b1[i];
+            sb3[i] = a.b3[i];
+        }
+        for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i] + 1.0f) * (1.0f / 3.0f);
+        for (int i = threadIdx.x; i < 256; i += kChainTcThreads) sWsig[i] = a.Wsig[i];
+        if (threadIdx.x < 16) {
+            sbmu[threadIdx.x] = a.bmu[threadIdx.x];
+            sbsig[threadIdx.x] = a.bsig[threadIdx.x];
+            sz0[threadIdx.x] = a.z0[threadIdx.x];
+        }
+        if (threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(bar_z, kChainEpiWarps);
+        mbar_init(bar_p, 1);
+        mbar_init(bar_h, kChainEpiWarps);
+        mbar_init(bar_h + 8, kChainEpiWarps);
+        mbar_init(bar_hfree, 1);
+        mbar_init(bar_hfree + 8, 1);
+        mbar_init(bar_acc2, 1);
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    fence_proxy_async();          // the operand image was written with ordinary stores; the MMAs read it asynchronously
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_tiles = ceil_div(a.count, 128);
+    const int n_phases = W + 2;                                   // W guide steps, transition, emission hidden layer
+
+    if (warp == 0) {
+        // ---------------- MMA issuer -------------------------------------------------------------------
+        const uint32_t idesc_h = instr_desc_tf32(H), idesc_mu = instr_desc_tf32(16), idesc_head = instr_desc_tf32(32);
+        uint32_t nz = 0, nu = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+            for (int ph = 0; ok && ph < n_phases; ++ph) {
+                ok = mbar_wait(bar_z, nz & 1u, abort_flag, a.st);
+                if (!ok) break;
+                ++nz;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t b_tile = ph < W ? t_zw1 : (ph == W ? t_zw1 + 64u : t_w3);
+                    const uint64_t a_desc = make_smem_desc(t_z), b_desc = make_smem_desc(b_tile);
+                    umma_tf32(tmem_base, a_desc, b_desc, idesc_h, 0u);
+                    umma_tf32(tmem_base, a_desc + 2, b_desc + 2, idesc_h, 1u);
+                    umma_commit(bar_p);
+                }
+                __syncwarp();
+                if (ph > W) continue;                              // the emission hidden layer has no second GEMM here
+                const uint32_t b_base = ph < W ? t_wmu : t_w2;
+                const uint32_t slab = ph < W ? 16u * 128u : 32u * 128u;
+                const uint32_t d_col = tmem_base + (ph < W ? kColMu : kColHead);
+                const uint32_t idesc2 = ph < W ? idesc_mu : idesc_head;
+                for (int c = 0; c < n_chunks; ++c, ++nu) {
+                    const uint32_t b = nu & 1u;
+                    ok = mbar_wait(bar_h + 8 * b, (nu >> 1) & 1u, abort_flag, a.st);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (lane == 0) {
+#pragma unroll
+                        for (int kb = 0; kb < 2; ++kb) {
+                            const uint64_t a_desc = make_smem_desc(t_hb + b * 32768u + kb * 16384u);
+                            const uint64_t b_desc = make_smem_desc(b_base + (2 * c + kb) * slab);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k)
+                                umma_tf32(d_col, a_desc + 2 * k, b_desc + 2 * k, idesc2, (c | kb | k) != 0 ? 1u : 0u);
+                        }
+                        umma_commit(bar_hfree + 8 * b);
+                        if (c == n_chunks - 1) umma_commit(bar_acc2);
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+        if (!ok) {
+            if (lane == 0) umma_commit(bar_drain);
+            __syncwarp();
+            mbar_wait_quiet(bar_drain, 0u);
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue ---------------------------------------------------------------------
+        const int q = warp & 3, cg = (warp - 1) >> 2;
+        const int row = q * 32 + lane;                                            // TMEM lane = sample of the tile
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        const uint32_t step = a.st->step;
+        uint32_t np = 0, na = 0, nu = 0;
+        bool ok = true;
+        (void)kblocks;
+        for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+            const int k = tile * 128 + row;
+            const uint32_t sample = a.sample_base + static_cast<uint32_t>(k);
+            // initial latent z_{T-l-1}
+            st_shared_v4(t_z + sw128(row, cg), tf32_rna(sz0[4 * cg + 0]), tf32_rna(sz0[4 * cg + 1]),
+                         tf32_rna(sz0[4 * cg + 2]), tf32_rna(sz0[4 * cg + 3]));
+            fence_proxy_async();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_z);
+
+            for (int ph = 0; ok && ph < n_phases; ++ph) {
+                ok = mbar_wait(bar_p, np & 1u, abort_flag, a.st);
+                if (!ok) break;
+                ++np;
+                tc_fence_after();
+                const float* bias = ph < W ? sbzs : (ph == W ? sb1 : sb3);
+                const float* lr = slr + (ph < W ? ph : 0) * H;
+                for (int c = 0; c < n_chunks; ++c) {
+                    const int col0 = c * 64 + cg * 16;
+                    uint32_t acc[16];
+                    tmem_ld16(lane_base + col0, acc);
+                    tmem_ld_wait();
+                    float h[16], bv[16];
+#pragma unroll
+                    for (int i4 = 0; i4 < 4; ++i4) {
+                        const float4 t4 = *reinterpret_cast<const float4*>(bias + col0 + 4 * i4);
+                        bv[4 * i4 + 0] = t4.x; bv[4 * i4 + 1] = t4.y; bv[4 * i4 + 2] = t4.z; bv[4 * i4 + 3] = t4.w;
+                    }
+                    if (ph < W) {
+                        float lv[16];
+#pragma unroll
+                        for (int i4 = 0; i4 < 4; ++i4) {
+                            const float4 t4 = *reinterpret_cast<const float4*>(lr + col0 + 4 * i4);
+                            lv[4 * i4 + 0] = t4.x; lv[4 * i4 + 1] = t4.y; lv[4 * i4 + 2] = t4.z; lv[4 * i4 + 3] = t4.w;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {            // tanh, then (tanh + h_left + h_right) / 3
+                            float e, r;
+                            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
+                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+                            h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) h[i] = fmaxf(__uint_as_float(acc[i]) + bv[i], 0.0f);
+                    }
+                    if (ph <= W) {
+                        const uint32_t b = nu & 1u;
+                        if (nu >= 2) {                            // the buffer's previous contents must have been multiplied
+                            ok = mbar_wait(bar_hfree + 8 * b, ((nu >> 1) - 1u) & 1u, abort_flag, a.st);
+                            if (!ok) break;
+                        }
+                        const uint32_t dst = t_hb + b * 32768u + static_cast<uint32_t>(cg >> 1) * 16384u;
+                        const int ch0 = (cg & 1) * 4;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            st_shared_v4(dst + sw128(row, ch0 + i), tf32_rna(h[4 * i + 0]), tf32_rna(h[4 * i + 1]),
+                                         tf32_rna(h[4 * i + 2]), tf32_rna(h[4 * i + 3]));
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(bar_h + 8 * b);
+                        ++nu;
+                    } else if (k < a.count) {
+                        float4* out = reinterpret_cast<float4*>(a.v_out + static_cast<size_t>(k) * H + col0);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            float4 o = make_float4(h[4 * i + 0], h[4 * i + 1], h[4 * i + 2], h[4 * i + 3]);
+                            if (a.round_v) { o.x = tf32_rna(o.x); o.y = tf32_rna(o.y); o.z = tf32_rna(o.z); o.w = tf32_rna(o.w); }
+                            out[i] = o;
+                        }
+                    }
+                }
+                if (!ok || ph > W) continue;
+
+                // ---- second result: the next latent ----------------------------------------------------
+                ok = mbar_wait(bar_acc2, na & 1u, abort_flag, a.st);
+                if (!ok) break;
+                ++na;
+                tc_fence_after();
+                float z_own[4];
+                if (ph < W) {
+                    uint32_t mu_bits[16];
+                    tmem_ld16(lane_base + kColMu, mu_bits);
+                    tmem_ld_wait();
+                    float mu[16];
+#pragma unroll
+                    for (int d = 0; d < 16; ++d) mu[d] = __uint_as_float(mu_bits[d]) + sbmu[d];
+                    float eps[4];
+                    normal4_fast(static_cast<uint32_t>(cg), sample, static_cast<uint32_t>(ph), step, a.key.seed_lo, a.key.seed_hi, eps);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const float* wrow = sWsig + (4 * cg + c) * 16;
+                        float pre = sbsig[4 * cg + c];
+#pragma unroll
+                        for (int e = 0; e < 16; ++e) pre = fmaf(wrow[e], mu[e], pre);
+                        float own = 0.0f;
+#pragma unroll
+                        for (int gg = 0; gg < 4; ++gg)
+                            if (gg == cg) own = mu[4 * gg + c];
+                        z_own[c] = fmaf(softplus_fast(pre), eps[c], own);
+                    }
+                } else {
+                    uint32_t mean_bits[16], lv_bits[16];
+                    tmem_ld16(lane_base + kColHead, mean_bits);
+                    tmem_ld16(lane_base + kColHead + 16, lv_bits);
+                    tmem_ld_wait();
+                    float eps[4];
+                    normal4_fast(static_cast<uint32_t>(cg), sample, kStreamTransition, step, a.key.seed_lo, a.key.seed_hi, eps);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float mean = 0.0f, lv = 0.0f;
+#pragma unroll
+                        for (int gg = 0; gg < 4; ++gg)
+                            if (gg == cg) { mean = __uint_as_float(mean_bits[4 * gg + c]); lv = __uint_as_float(lv_bits[4 * gg + c]); }
+                        z_own[c] = fmaf(exp_half_fast(lv + sb2[16 + 4 * cg + c]), eps[c], mean + sb2[4 * cg + c]);
+                    }
+                }
+                st_shared_v4(t_z + sw128(row, cg), tf32_rna(z_own[0]), tf32_rna(z_own[1]), tf32_rna(z_own[2]), tf32_rna(z_own[3]));
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_z);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+}  // namespace tc
+}  // namespace cutoff

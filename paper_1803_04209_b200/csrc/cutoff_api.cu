@@ -12,6 +12,7 @@
 #include "kernels_model.cuh"
 #include "kernels_sort.cuh"
 #include "emit_tc.cuh"
+#include "chain_tc.cuh"
 
 using namespace cutoff;
 
@@ -60,6 +61,8 @@ struct cutoff_ctx {
     CUtensorMap map_v{};            // TMA view of d_v   [alloc_rows][H]
     CUtensorMap map_w4{};           // TMA view of W4    [2N][H]
     bool use_tc = false;            // emission output layer on tensor cores
+    bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
+    float* d_chain_image = nullptr; // swizzled tf32 operand tiles of the chain
 
     float* h_stage = nullptr;       // pinned [N]
     DevState* h_state = nullptr;    // pinned
@@ -112,7 +115,7 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
-    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_ring); cudaFree(c->d_stage);
+    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_chain_image); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
     cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
     if (c->h_stage) cudaFreeHost(c->h_stage);
@@ -198,7 +201,27 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
     }
 }
 
+void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(tc::k_chain_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        attr_set = true;
+    }
+    tc::ChainTcArgs a;
+    const ModelDev& m = c->m;
+    a.image = c->d_chain_image;
+    a.bz = m.bz; a.b1 = m.b1; a.b3 = m.b3; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig; a.b2 = m.b2; a.z0 = m.z0;
+    a.hlr = c->d_hlr; a.st = c->d_state;
+    a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.round_v = 1; a.v_out = c->d_v;
+    const int tiles = ceil_div(count, 128);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    tc::k_chain_tc<<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W), c->stream>>>(a);
+    c->launches += 1;
+}
+
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
+    if (c->chain_tc) { launch_chain_tc(c, sample_base, count); return; }
     const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
     switch (c->D) {
         case 4: launch_chain_t<4>(c, sample_base, count, smem); break;
@@ -424,11 +447,14 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     if (ceil_div(c->S, kMaxChunks) > c->alloc_rows) return fail(CUTOFF_ERR_UNSUPPORTED);   // S too large for the pass buffers
     plan_chunks(c, c->alloc_rows);
     c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
+    c->chain_tc = c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
+                  tc::chain_tc_smem_bytes(c->H, c->W) <= 227 * 1024;
 
     size_t blob_floats = 0;
     for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
     CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
     CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 3 * c->H * c->D));
+    if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_state, sizeof(DevState)));
@@ -508,6 +534,43 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
             for (size_t d = 0; d < D; ++d) wT[t * H * D + d * H + i] = w[i * D + d];
     }
     CU_CHECK(c, cudaMemcpy(c->d_WT, wT.data(), wT.size() * sizeof(float), cudaMemcpyHostToDevice));
+
+    if (c->chain_tc) {
+        // Operand tiles of the tensor-core chain as they will sit in shared memory: tf32 (nearest, ties
+        // away), K-major rows of 32 values, 16-byte chunks XOR-swizzled with the row index modulo 8.
+        auto tf32 = [](float f) {
+            uint32_t u;
+            std::memcpy(&u, &f, 4);
+            u = (u + 0x1000u) & 0xFFFFE000u;
+            std::memcpy(&f, &u, 4);
+            return f;
+        };
+        auto at = [](size_t row, size_t col) {       // float index inside one slab of rows x 32
+            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
+        };
+        std::vector<float> img(tc::chain_tc_image_floats(c->H), 0.0f);
+        const float* wz = host.data() + off[8];      // [H][D]
+        const float* w1 = host.data() + off[15];     // [H][D]
+        const float* w3 = host.data() + off[19];     // [H][D]
+        const float* wmu = host.data() + off[10];    // [D][H]
+        const float* w2 = host.data() + off[17];     // [2D][H]
+        float* t_zw1 = img.data();
+        float* t_w3 = t_zw1 + H * 32;
+        float* t_wmu = t_w3 + H * 32;
+        float* t_w2 = t_wmu + H * 16;
+        for (size_t n = 0; n < H; ++n)
+            for (size_t k = 0; k < D; ++k) {
+                t_zw1[at(n, k)] = tf32(wz[n * D + k]);
+                t_zw1[at(n, 16 + k)] = tf32(w1[n * D + k]);
+                t_w3[at(n, k)] = tf32(w3[n * D + k]);
+            }
+        for (size_t kb = 0; kb < H / 32; ++kb)
+            for (size_t jj = 0; jj < 32; ++jj) {
+                for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
+                for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + at(o, jj)] = tf32(w2[o * H + kb * 32 + jj]);
+            }
+        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
 
     ModelDev& m = c->m;
     m.N = c->N; m.D = c->D; m.H = c->H; m.W = c->W;
