@@ -31,7 +31,14 @@ if ROOT not in sys.path:
 METRIC = "predicted_worker_times_per_sec"
 UNIT = "worker-times/s"
 SM_COUNT = 148
-FP32_LANES_PER_SM = 128
+FP32_LANES_PER_SM = 128          # fused multiply-add lanes per SM per clock
+MINMAX_LANES_PER_SM = 64         # fp32 min / max lanes per SM per clock (ALU pipe: 16 per sub-partition)
+# DRAM bytes per launch of the dominant kernel, from the ncu capture summarised under profiles/ (valid for the
+# kernel as committed with that summary; set to None when the kernel changes).
+NCU_TRAFFIC = {
+    ("n1024", "sort"): {"bytes_per_sample": 201550848 / 49152 + 4397312 / 49152,
+                        "source": "profiles/ncu_full_n1024_s49152_chain_emit_sort.txt (S=49152, scaled by S)"},
+}
 PRECISION_NAMES = {0: "f32", 1: "tf32", 2: "tf32(bf16 weights)"}
 
 
@@ -314,19 +321,26 @@ def main():
     dominant = max(stage_avg, key=stage_avg.get)
     kind, amount = work[dominant]
     dur = stage_avg[dominant] * 1e-3
+    smax = peaks.get("sm_max_mhz", 1965.0)
     if kind == "tensor":
         bf16 = peaks.get("bf16_tflops", 1590.0)
         peak, unit = 0.5 * bf16, "TFLOP/s"             # tf32 runs at half the bf16 rate (nominal ratio)
         peak_src = ("measured bf16 burst x 0.5 (nominal tf32 : bf16 ratio)" if peaks else "fallback 1590 x 0.5")
         bound = "tensor"
+    elif dominant == "sort":
+        peak, unit = SM_COUNT * MINMAX_LANES_PER_SM * smax * 1e6 / 1e12, "Tlane-op/s"
+        peak_src = "148 SMs x 64 fp32 min/max lanes x max SM clock"
+        bound = "alu"
     else:
-        smax = peaks.get("sm_max_mhz", 1965.0)
         peak, unit = SM_COUNT * FP32_LANES_PER_SM * smax * 1e6 / 1e12, "Tlane-op/s"
         peak_src = "148 SMs x 128 fp32 lanes x max SM clock"
         bound = "alu"
     achieved = amount / dur / 1e12
+    traffic = NCU_TRAFFIC.get((wl.name, dominant))
     roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": None, "peak_source": peak_src,
+                "frac": achieved / peak, "traffic": traffic["bytes_per_sample"] * wl.S if traffic else None,
+                "traffic_source": traffic["source"] if traffic else None,
+                "algorithmic_per_launch": amount, "peak_source": peak_src,
                 "stage_ms": {k: round(v, 4) for k, v in stage_avg.items()}}
 
     cpu_baseline = None
