@@ -30,7 +30,6 @@ namespace tc {
 constexpr int kChainEpiWarps = 16;
 constexpr int kChainTcThreads = (1 + kChainEpiWarps) * 32;
 constexpr int kChainD = 16;
-constexpr int kColMu = 256, kColHead = 320;      // TMEM columns of the second-GEMM results
 
 struct ChainTcArgs {
     const float* image;         // swizzled operand tiles: [Wz|W1] (H x 32), W3 (H x 32), Wmu (H/32 x 16 x 32), W2 (H/32 x 32 x 32)
@@ -46,7 +45,7 @@ struct ChainTcArgs {
 inline size_t chain_tc_image_floats(int H) { return static_cast<size_t>(H) * (32 + 32 + 16 + 32); }
 
 inline size_t chain_tc_smem_bytes(int H, int W) {
-    const size_t tiles = chain_tc_image_floats(H) * 4 + 128 * 128 + 2 * 2 * 128 * 128;
+    const size_t tiles = chain_tc_image_floats(H) * 4 + 2 * 128 * 128 /*Z x2*/ + 4 * 128 * 128 /*hidden chunks: 2 per slot*/;
     const size_t floats = 3 * static_cast<size_t>(H) + static_cast<size_t>(W) * H + 16 * 16 + 16 + 16 + 32 + 16;
     return 1024 + tiles + floats * 4 + 256;
 }
@@ -76,23 +75,33 @@ __device__ __forceinline__ float softplus_fast(float x) {          // ln(1 + e^x
     return x > 15.0f ? x : 0.6931471805599453f * __log2f(1.0f + e);
 }
 
+// One of the two tiles a CTA has in flight: its shared-memory operands, TMEM columns and barriers,
+// and how many times each barrier has completed (both roles count the same sequence).
+struct ChainSlot {
+    uint32_t t_z;            // latent A operand [128 x 128 B]
+    uint32_t t_hb;           // two hidden-chunk A operands [128 x 128 B] each
+    uint32_t tmem;           // first of the slot's 256 TMEM columns
+    uint32_t bar_z, bar_p, bar_h, bar_hfree, bar_acc2;     // bar_h, bar_hfree: two barriers each
+    uint32_t nz, np, na, nu;
+    int tile;                // current tile, -1 if the slot is idle
+};
+
 __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const int H = a.H, W = a.W;
-    const int n_chunks = H / 64, kblocks = H / 32;
+    const int n_chunks = H / 32;                                  // a chunk = 32 hidden units = one K block
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (base - raw);
-    // operand tiles
+    // weight operand tiles
     const uint32_t t_zw1 = base;
     const uint32_t t_w3 = t_zw1 + H * 128;
     const uint32_t t_wmu = t_w3 + H * 128;
     const uint32_t t_w2 = t_wmu + H * 64;
-    const uint32_t t_z = t_w2 + H * 128;
-    const uint32_t t_hb = t_z + 128 * 128;                       // two buffers of 32 KB
     const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u;
+    const uint32_t t_act = base + image_bytes;                    // Z0, Z1, then 4 hidden-chunk buffers: 6 x 16 KB
     // fp32 side tables
-    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 128 * 128 + 2 * 32768);    // bz * 2 log2(e)
+    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz * 2 log2(e)
     float* sb1 = sbzs + H;
     float* sb3 = sb1 + H;
     float* slr = sb3 + H;                    // [W][H]  (h_left + h_right + 1) / 3
@@ -101,11 +110,10 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     float* sbsig = sbmu + 16;
     float* sb2 = sbsig + 16;                 // [32]
     float* sz0 = sb2 + 32;                   // [16]
-    const uint32_t bars = smem_u32(sz0 + 16);
-    const uint32_t bar_z = bars, bar_p = bars + 8, bar_h = bars + 16 /*2*/, bar_hfree = bars + 32 /*2*/,
-                   bar_acc2 = bars + 48, bar_drain = bars + 56;
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sz0 + 16 + 16);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sz0 + 16 + 18);
+    const uint32_t bars = smem_u32(sz0 + 16);                     // 2 slots x 7 barriers, then the drain barrier
+    const uint32_t bar_drain = bars + 2 * 56;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sz0 + 16 + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sz0 + 16 + 34);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -129,13 +137,16 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         if (threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
     }
     if (threadIdx.x == 0) {
-        mbar_init(bar_z, kChainEpiWarps);
-        mbar_init(bar_p, 1);
-        mbar_init(bar_h, kChainEpiWarps);
-        mbar_init(bar_h + 8, kChainEpiWarps);
-        mbar_init(bar_hfree, 1);
-        mbar_init(bar_hfree + 8, 1);
-        mbar_init(bar_acc2, 1);
+        for (uint32_t s = 0; s < 2; ++s) {
+            const uint32_t b0 = bars + 56 * s;
+            mbar_init(b0, kChainEpiWarps);           // z ready
+            mbar_init(b0 + 8, 1);                    // hidden pre-activations ready
+            mbar_init(b0 + 16, kChainEpiWarps);      // hidden chunk buffer 0 written
+            mbar_init(b0 + 24, kChainEpiWarps);      // hidden chunk buffer 1 written
+            mbar_init(b0 + 32, 1);                   // hidden chunk buffer 0 multiplied
+            mbar_init(b0 + 40, 1);                   // hidden chunk buffer 1 multiplied
+            mbar_init(b0 + 48, 1);                   // second result ready
+        }
         mbar_init(bar_drain, 1);
         *abort_flag = 0;
         fence_barrier_init();
@@ -151,51 +162,72 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    ChainSlot slot[2];
+#pragma unroll
+    for (uint32_t s = 0; s < 2; ++s) {
+        const uint32_t b0 = bars + 56 * s;
+        slot[s].t_z = t_act + s * 16384u;
+        slot[s].t_hb = t_act + 2 * 16384u + s * 32768u;
+        slot[s].tmem = tmem_base + s * 256u;
+        slot[s].bar_z = b0; slot[s].bar_p = b0 + 8; slot[s].bar_h = b0 + 16; slot[s].bar_hfree = b0 + 32;
+        slot[s].bar_acc2 = b0 + 48;
+        slot[s].nz = slot[s].np = slot[s].na = slot[s].nu = 0;
+        slot[s].tile = -1;
+    }
     const int n_tiles = ceil_div(a.count, 128);
     const int n_phases = W + 2;                                   // W guide steps, transition, emission hidden layer
+    // The second result of a tile (mu: 16 columns, mean | logvar: 32 columns) reuses the first columns of the
+    // tile's pre-activation block: those are multiplied only after every warp has read chunk 0.
 
     if (warp == 0) {
         // ---------------- MMA issuer -------------------------------------------------------------------
         const uint32_t idesc_h = instr_desc_tf32(H), idesc_mu = instr_desc_tf32(16), idesc_head = instr_desc_tf32(32);
-        uint32_t nz = 0, nu = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
+        for (int t0 = blockIdx.x; ok && t0 < n_tiles; t0 += 2 * gridDim.x) {
+            slot[0].tile = t0;
+            slot[1].tile = t0 + static_cast<int>(gridDim.x) < n_tiles ? t0 + static_cast<int>(gridDim.x) : -1;
             for (int ph = 0; ok && ph < n_phases; ++ph) {
-                ok = mbar_wait(bar_z, nz & 1u, abort_flag, a.st);
-                if (!ok) break;
-                ++nz;
-                tc_fence_after();
-                if (lane == 0) {
-                    const uint32_t b_tile = ph < W ? t_zw1 : (ph == W ? t_zw1 + 64u : t_w3);
-                    const uint64_t a_desc = make_smem_desc(t_z), b_desc = make_smem_desc(b_tile);
-                    umma_tf32(tmem_base, a_desc, b_desc, idesc_h, 0u);
-                    umma_tf32(tmem_base, a_desc + 2, b_desc + 2, idesc_h, 1u);
-                    umma_commit(bar_p);
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {                       // first GEMM of both tiles
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    ok = mbar_wait(sl.bar_z, sl.nz & 1u, abort_flag, a.st);
+                    if (!ok) continue;
+                    ++sl.nz;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t b_tile = ph < W ? t_zw1 : (ph == W ? t_zw1 + 64u : t_w3);
+                        const uint64_t a_desc = make_smem_desc(sl.t_z), b_desc = make_smem_desc(b_tile);
+                        umma_tf32(sl.tmem, a_desc, b_desc, idesc_h, 0u);
+                        umma_tf32(sl.tmem, a_desc + 2, b_desc + 2, idesc_h, 1u);
+                        umma_commit(sl.bar_p);
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
                 if (ph > W) continue;                              // the emission hidden layer has no second GEMM here
                 const uint32_t b_base = ph < W ? t_wmu : t_w2;
                 const uint32_t slab = ph < W ? 16u * 128u : 32u * 128u;
-                const uint32_t d_col = tmem_base + (ph < W ? kColMu : kColHead);
                 const uint32_t idesc2 = ph < W ? idesc_mu : idesc_head;
-                for (int c = 0; c < n_chunks; ++c, ++nu) {
-                    const uint32_t b = nu & 1u;
-                    ok = mbar_wait(bar_h + 8 * b, (nu >> 1) & 1u, abort_flag, a.st);
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (lane == 0) {
 #pragma unroll
-                        for (int kb = 0; kb < 2; ++kb) {
-                            const uint64_t a_desc = make_smem_desc(t_hb + b * 32768u + kb * 16384u);
-                            const uint64_t b_desc = make_smem_desc(b_base + (2 * c + kb) * slab);
+                for (int s = 0; s < 2; ++s) {                       // second GEMM, chunk by chunk as the epilogue delivers
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    for (int c = 0; c < n_chunks; ++c, ++sl.nu) {
+                        const uint32_t b = sl.nu & 1u;
+                        ok = mbar_wait(sl.bar_h + 8 * b, (sl.nu >> 1) & 1u, abort_flag, a.st);
+                        if (!ok) break;
+                        tc_fence_after();
+                        if (lane == 0) {
+                            const uint64_t a_desc = make_smem_desc(sl.t_hb + b * 16384u);
+                            const uint64_t b_desc = make_smem_desc(b_base + c * slab);
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
-                                umma_tf32(d_col, a_desc + 2 * k, b_desc + 2 * k, idesc2, (c | kb | k) != 0 ? 1u : 0u);
+                                umma_tf32(sl.tmem, a_desc + 2 * k, b_desc + 2 * k, idesc2, (c | k) != 0 ? 1u : 0u);
+                            umma_commit(sl.bar_hfree + 8 * b);
+                            if (c == n_chunks - 1) umma_commit(sl.bar_acc2);
                         }
-                        umma_commit(bar_hfree + 8 * b);
-                        if (c == n_chunks - 1) umma_commit(bar_acc2);
+                        __syncwarp();
                     }
-                    __syncwarp();
                 }
             }
         }
@@ -209,134 +241,140 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         // ---------------- epilogue ---------------------------------------------------------------------
         const int q = warp & 3, cg = (warp - 1) >> 2;
         const int row = q * 32 + lane;                                            // TMEM lane = sample of the tile
-        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t step = a.st->step;
-        uint32_t np = 0, na = 0, nu = 0;
         bool ok = true;
-        (void)kblocks;
-        for (int tile = blockIdx.x; ok && tile < n_tiles; tile += gridDim.x) {
-            const int k = tile * 128 + row;
-            const uint32_t sample = a.sample_base + static_cast<uint32_t>(k);
-            // initial latent z_{T-l-1}
-            st_shared_v4(t_z + sw128(row, cg), tf32_rna(sz0[4 * cg + 0]), tf32_rna(sz0[4 * cg + 1]),
-                         tf32_rna(sz0[4 * cg + 2]), tf32_rna(sz0[4 * cg + 3]));
-            fence_proxy_async();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(bar_z);
-
+        for (int t0 = blockIdx.x; ok && t0 < n_tiles; t0 += 2 * gridDim.x) {
+            slot[0].tile = t0;
+            slot[1].tile = t0 + static_cast<int>(gridDim.x) < n_tiles ? t0 + static_cast<int>(gridDim.x) : -1;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {                           // initial latent z_{T-l-1} of both tiles
+                if (slot[s].tile < 0) continue;
+                st_shared_v4(slot[s].t_z + sw128(row, cg), tf32_rna(sz0[4 * cg + 0]), tf32_rna(sz0[4 * cg + 1]),
+                             tf32_rna(sz0[4 * cg + 2]), tf32_rna(sz0[4 * cg + 3]));
+                fence_proxy_async();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(slot[s].bar_z);
+            }
             for (int ph = 0; ok && ph < n_phases; ++ph) {
-                ok = mbar_wait(bar_p, np & 1u, abort_flag, a.st);
-                if (!ok) break;
-                ++np;
-                tc_fence_after();
                 const float* bias = ph < W ? sbzs : (ph == W ? sb1 : sb3);
                 const float* lr = slr + (ph < W ? ph : 0) * H;
-                for (int c = 0; c < n_chunks; ++c) {
-                    const int col0 = c * 64 + cg * 16;
-                    uint32_t acc[16];
-                    tmem_ld16(lane_base + col0, acc);
-                    tmem_ld_wait();
-                    float h[16], bv[16];
+                // ---- hidden layer of both tiles: bias, activation, next A operand (or v) -----------------
 #pragma unroll
-                    for (int i4 = 0; i4 < 4; ++i4) {
-                        const float4 t4 = *reinterpret_cast<const float4*>(bias + col0 + 4 * i4);
-                        bv[4 * i4 + 0] = t4.x; bv[4 * i4 + 1] = t4.y; bv[4 * i4 + 2] = t4.z; bv[4 * i4 + 3] = t4.w;
-                    }
-                    if (ph < W) {
-                        float lv[16];
+                for (int s = 0; s < 2; ++s) {
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    ok = mbar_wait(sl.bar_p, sl.np & 1u, abort_flag, a.st);
+                    if (!ok) continue;
+                    ++sl.np;
+                    tc_fence_after();
+                    const int k = sl.tile * 128 + row;
+                    for (int c = 0; c < n_chunks; ++c) {
+                        const int col0 = c * 32 + cg * 8;
+                        uint32_t acc[8];
+                        tmem_ld8(sl.tmem + lane_off + col0, acc);
+                        tmem_ld_wait();
+                        const float4 b_lo = *reinterpret_cast<const float4*>(bias + col0);
+                        const float4 b_hi = *reinterpret_cast<const float4*>(bias + col0 + 4);
+                        const float bv[8] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w, b_hi.x, b_hi.y, b_hi.z, b_hi.w};
+                        float h[8];
+                        if (ph < W) {
+                            const float4 l_lo = *reinterpret_cast<const float4*>(lr + col0);
+                            const float4 l_hi = *reinterpret_cast<const float4*>(lr + col0 + 4);
+                            const float lv[8] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
 #pragma unroll
-                        for (int i4 = 0; i4 < 4; ++i4) {
-                            const float4 t4 = *reinterpret_cast<const float4*>(lr + col0 + 4 * i4);
-                            lv[4 * i4 + 0] = t4.x; lv[4 * i4 + 1] = t4.y; lv[4 * i4 + 2] = t4.z; lv[4 * i4 + 3] = t4.w;
+                            for (int i = 0; i < 8; ++i) {          // tanh, then (tanh + h_left + h_right) / 3
+                                float e, r;
+                                asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
+                                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+                                h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                            }
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) h[i] = fmaxf(__uint_as_float(acc[i]) + bv[i], 0.0f);
                         }
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {            // tanh, then (tanh + h_left + h_right) / 3
-                            float e, r;
-                            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
-                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-                            h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
-                        }
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) h[i] = fmaxf(__uint_as_float(acc[i]) + bv[i], 0.0f);
-                    }
-                    if (ph <= W) {
-                        const uint32_t b = nu & 1u;
-                        if (nu >= 2) {                            // the buffer's previous contents must have been multiplied
-                            ok = mbar_wait(bar_hfree + 8 * b, ((nu >> 1) - 1u) & 1u, abort_flag, a.st);
-                            if (!ok) break;
-                        }
-                        const uint32_t dst = t_hb + b * 32768u + static_cast<uint32_t>(cg >> 1) * 16384u;
-                        const int ch0 = (cg & 1) * 4;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i)
-                            st_shared_v4(dst + sw128(row, ch0 + i), tf32_rna(h[4 * i + 0]), tf32_rna(h[4 * i + 1]),
-                                         tf32_rna(h[4 * i + 2]), tf32_rna(h[4 * i + 3]));
-                        fence_proxy_async();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(bar_h + 8 * b);
-                        ++nu;
-                    } else if (k < a.count) {
-                        float4* out = reinterpret_cast<float4*>(a.v_out + static_cast<size_t>(k) * H + col0);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            float4 o = make_float4(h[4 * i + 0], h[4 * i + 1], h[4 * i + 2], h[4 * i + 3]);
-                            if (a.round_v) { o.x = tf32_rna(o.x); o.y = tf32_rna(o.y); o.z = tf32_rna(o.z); o.w = tf32_rna(o.w); }
-                            out[i] = o;
+                        if (ph <= W) {
+                            const uint32_t b = sl.nu & 1u;
+                            if (sl.nu >= 2) {                      // the buffer's previous contents must have been multiplied
+                                ok = mbar_wait(sl.bar_hfree + 8 * b, ((sl.nu >> 1) - 1u) & 1u, abort_flag, a.st);
+                                if (!ok) break;
+                            }
+                            const uint32_t dst = sl.t_hb + b * 16384u;
+                            st_shared_v4(dst + sw128(row, 2 * cg), tf32_rna(h[0]), tf32_rna(h[1]), tf32_rna(h[2]), tf32_rna(h[3]));
+                            st_shared_v4(dst + sw128(row, 2 * cg + 1), tf32_rna(h[4]), tf32_rna(h[5]), tf32_rna(h[6]), tf32_rna(h[7]));
+                            fence_proxy_async();
+                            tc_fence_before();                     // our TMEM reads of this chunk precede the MMAs it unblocks
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(sl.bar_h + 8 * b);
+                            ++sl.nu;
+                        } else if (k < a.count) {
+                            float4* out = reinterpret_cast<float4*>(a.v_out + static_cast<size_t>(k) * H + col0);
+                            float4 o0 = make_float4(h[0], h[1], h[2], h[3]), o1 = make_float4(h[4], h[5], h[6], h[7]);
+                            if (a.round_v) {
+                                o0.x = tf32_rna(o0.x); o0.y = tf32_rna(o0.y); o0.z = tf32_rna(o0.z); o0.w = tf32_rna(o0.w);
+                                o1.x = tf32_rna(o1.x); o1.y = tf32_rna(o1.y); o1.z = tf32_rna(o1.z); o1.w = tf32_rna(o1.w);
+                            }
+                            out[0] = o0;
+                            out[1] = o1;
                         }
                     }
                 }
                 if (!ok || ph > W) continue;
-
-                // ---- second result: the next latent ----------------------------------------------------
-                ok = mbar_wait(bar_acc2, na & 1u, abort_flag, a.st);
-                if (!ok) break;
-                ++na;
-                tc_fence_after();
-                float z_own[4];
-                if (ph < W) {
-                    uint32_t mu_bits[16];
-                    tmem_ld16(lane_base + kColMu, mu_bits);
-                    tmem_ld_wait();
-                    float mu[16];
+                // ---- second result of both tiles: the next latent -----------------------------------------
 #pragma unroll
-                    for (int d = 0; d < 16; ++d) mu[d] = __uint_as_float(mu_bits[d]) + sbmu[d];
-                    float eps[4];
-                    normal4_fast(static_cast<uint32_t>(cg), sample, static_cast<uint32_t>(ph), step, a.key.seed_lo, a.key.seed_hi, eps);
+                for (int s = 0; s < 2; ++s) {
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    ok = mbar_wait(sl.bar_acc2, sl.na & 1u, abort_flag, a.st);
+                    if (!ok) continue;
+                    ++sl.na;
+                    tc_fence_after();
+                    const uint32_t sample = a.sample_base + static_cast<uint32_t>(sl.tile * 128 + row);
+                    float z_own[4];
+                    if (ph < W) {
+                        uint32_t mu_bits[16];
+                        tmem_ld16(sl.tmem + lane_off, mu_bits);
+                        tmem_ld_wait();
+                        float mu[16];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const float* wrow = sWsig + (4 * cg + c) * 16;
-                        float pre = sbsig[4 * cg + c];
+                        for (int d = 0; d < 16; ++d) mu[d] = __uint_as_float(mu_bits[d]) + sbmu[d];
+                        float eps[4];
+                        normal4_fast(static_cast<uint32_t>(cg), sample, static_cast<uint32_t>(ph), step, a.key.seed_lo, a.key.seed_hi, eps);
 #pragma unroll
-                        for (int e = 0; e < 16; ++e) pre = fmaf(wrow[e], mu[e], pre);
-                        float own = 0.0f;
+                        for (int c = 0; c < 4; ++c) {
+                            const float* wrow = sWsig + (4 * cg + c) * 16;
+                            float pre = sbsig[4 * cg + c];
 #pragma unroll
-                        for (int gg = 0; gg < 4; ++gg)
-                            if (gg == cg) own = mu[4 * gg + c];
-                        z_own[c] = fmaf(softplus_fast(pre), eps[c], own);
+                            for (int e = 0; e < 16; ++e) pre = fmaf(wrow[e], mu[e], pre);
+                            float own = 0.0f;
+#pragma unroll
+                            for (int gg = 0; gg < 4; ++gg)
+                                if (gg == cg) own = mu[4 * gg + c];
+                            z_own[c] = fmaf(softplus_fast(pre), eps[c], own);
+                        }
+                    } else {
+                        uint32_t mean_bits[16], lv_bits[16];
+                        tmem_ld16(sl.tmem + lane_off, mean_bits);
+                        tmem_ld16(sl.tmem + lane_off + 16, lv_bits);
+                        tmem_ld_wait();
+                        float eps[4];
+                        normal4_fast(static_cast<uint32_t>(cg), sample, kStreamTransition, step, a.key.seed_lo, a.key.seed_hi, eps);
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            float mean = 0.0f, lv = 0.0f;
+#pragma unroll
+                            for (int gg = 0; gg < 4; ++gg)
+                                if (gg == cg) { mean = __uint_as_float(mean_bits[4 * gg + c]); lv = __uint_as_float(lv_bits[4 * gg + c]); }
+                            z_own[c] = fmaf(exp_half_fast(lv + sb2[16 + 4 * cg + c]), eps[c], mean + sb2[4 * cg + c]);
+                        }
                     }
-                } else {
-                    uint32_t mean_bits[16], lv_bits[16];
-                    tmem_ld16(lane_base + kColHead, mean_bits);
-                    tmem_ld16(lane_base + kColHead + 16, lv_bits);
-                    tmem_ld_wait();
-                    float eps[4];
-                    normal4_fast(static_cast<uint32_t>(cg), sample, kStreamTransition, step, a.key.seed_lo, a.key.seed_hi, eps);
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        float mean = 0.0f, lv = 0.0f;
-#pragma unroll
-                        for (int gg = 0; gg < 4; ++gg)
-                            if (gg == cg) { mean = __uint_as_float(mean_bits[4 * gg + c]); lv = __uint_as_float(lv_bits[4 * gg + c]); }
-                        z_own[c] = fmaf(exp_half_fast(lv + sb2[16 + 4 * cg + c]), eps[c], mean + sb2[4 * cg + c]);
-                    }
+                    st_shared_v4(sl.t_z + sw128(row, cg), tf32_rna(z_own[0]), tf32_rna(z_own[1]), tf32_rna(z_own[2]), tf32_rna(z_own[3]));
+                    fence_proxy_async();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sl.bar_z);
                 }
-                st_shared_v4(t_z + sw128(row, cg), tf32_rna(z_own[0]), tf32_rna(z_own[1]), tf32_rna(z_own[2]), tf32_rna(z_own[3]));
-                fence_proxy_async();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_z);
             }
         }
     }
