@@ -196,7 +196,7 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
         k_chain_resident<D><<<grid, kChainResidentThreads, resident, c->stream>>>(c->m, c->d_hlr, c->d_state, key,
                                                                                 sample_base, count, round_v, c->d_v);
     } else {
-        k_chain<D><<<ceil_div(count, ChainShape<D>::kSamplesPerCta), kChainThreads, smem, c->stream>>>(
+        k_chain<D><<<ceil_div(count, ChainShape<D>::kSamplesPerCta), ChainShape<D>::kThreads, smem, c->stream>>>(
             c->m, c->d_hlr, c->d_state, key, sample_base, count, round_v, c->d_v);
     }
 }

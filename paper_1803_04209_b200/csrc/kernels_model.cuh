@@ -232,12 +232,12 @@ inline size_t enc_rnn_resident_smem_floats(int H, int W) {
 // from consecutive addresses and all groups of a warp read as a broadcast.  Partial outputs are
 // summed over the group with xor-shuffles.  Each weight read serves all SPL samples of the lane.
 // ---------------------------------------------------------------------------------------------
-constexpr int kChainThreads = 128;
-
 template <int D> struct ChainShape {
     static constexpr int G = D / 4;                   // lanes per group
     static constexpr int SPL = D <= 16 ? 2 : 1;       // samples per lane
-    static constexpr int kSamplesPerCta = kChainThreads / G * SPL;
+    // threads of the phase-staged kernel: its shared memory allows one CTA per SM at D = 32, so that CTA is wide
+    static constexpr int kThreads = D <= 16 ? 128 : 384;
+    static constexpr int kSamplesPerCta = kThreads / G * SPL;
 };
 
 __device__ __forceinline__ float softplusf(float x) { return x > 20.0f ? x : log1pf(expf(x)); }
@@ -458,7 +458,7 @@ __device__ __forceinline__ void chain_emission_hidden(const ModelDev& m, const f
 
 // Variant 1: weights staged phase by phase (any model size whose largest phase fits in shared memory).
 template <int D>
-__global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float* __restrict__ hlr,
+__global__ void __launch_bounds__(ChainShape<D>::kThreads) k_chain(ModelDev m, const float* __restrict__ hlr,
                                                           const DevState* __restrict__ st, NoiseKey key,
                                                           uint32_t sample_base, int count, int round_v,
                                                           float* __restrict__ v_out /*[count][H]*/) {
@@ -466,7 +466,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float
     extern __shared__ __align__(16) float sm[];
     const int H = m.H, W = m.W;
     const int g = threadIdx.x % G;
-    const int k0 = (blockIdx.x * (kChainThreads / G) + threadIdx.x / G) * SPL;      // first sample of the lane
+    const int k0 = (blockIdx.x * (ChainShape<D>::kThreads / G) + threadIdx.x / G) * SPL;      // first sample of the lane
     const ChainNoise nz{key, st->step, sample_base + static_cast<uint32_t>(k0)};
 
     float* sWzT = sm;                   // [D][H]
@@ -478,7 +478,7 @@ __global__ void __launch_bounds__(kChainThreads) k_chain(ModelDev m, const float
     stage_vector4(sWmu, m.Wmu, H * D);
     stage_vector4(sWsig, m.Wsig, D * D);
     stage_vector4(sbz, m.bz, H);
-    for (int i = threadIdx.x; i < W * H; i += kChainThreads) shl[i] = hlr[i] + hlr[W * H + i];
+    for (int i = threadIdx.x; i < W * H; i += blockDim.x) shl[i] = hlr[i] + hlr[W * H + i];
     __syncthreads();
     float z[SPL][D];
 #pragma unroll
