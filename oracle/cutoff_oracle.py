@@ -61,6 +61,7 @@ _SH32 = np.uint64(32)
 
 STREAM_TRANSITION = 0x100       # guide step t uses stream t (0 .. lag)
 STREAM_EMISSION = 0x200
+STREAM_IMPUTE = 0x300           # where the scan for a censored worker's replacement starts
 
 
 def philox4x32_10(c0, c1, c2, c3, k0, k1):
@@ -252,6 +253,35 @@ def argmax_cutoff(omega: np.ndarray):
     return c_star, bool(best == -np.inf)
 
 
+def impute_censored(runtimes_sec, censored, predictive_sec, seed: int, step: int):
+    """Replace censored run-times by draws from the predictive distribution, left-truncated at the cutoff time.
+
+    Section 4.2 ("Handling Censored Run-times"): stragglers are killed once c gradients have arrived,
+    so their run-times are only known to exceed the cutoff time -- the largest run-time that was
+    observed in this step.  Each censored worker gets a draw from its own predictive distribution for
+    this step, p(x; x > cutoff time) = p(x) / P(x > cutoff time).  The predictive distribution is the
+    Monte-Carlo one: predictive_sec[k, j] is the k-th predictive draw of worker j (seconds).  The draws
+    are iid, so taking the first one above the threshold, scanning cyclically from a start index that
+    does not depend on their values, is an exact draw from the truncated distribution.  The start is
+    Philox word 0 of counter (worker, 0, STREAM_IMPUTE, step) modulo the number of draws.  If no draw of
+    a worker exceeds the threshold, the threshold itself is used (all that is known).
+    """
+    x = np.array(runtimes_sec, dtype=np.float64)
+    censored = np.asarray(censored).astype(bool)
+    if not censored.any():
+        return x, None
+    assert not censored.all(), "at least one worker must have finished"
+    threshold = float(x[~censored].max())
+    S = predictive_sec.shape[0]
+    for j in np.flatnonzero(censored):
+        word0 = int(philox4x32_10(int(j), 0, STREAM_IMPUTE, step, seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)[0])
+        start = word0 % S
+        column = np.roll(predictive_sec[:, j], -start)          # scan order: start, start+1, ..., wrapping
+        above = np.flatnonzero(column > threshold)
+        x[j] = column[above[0]] if above.size else threshold
+    return x, threshold
+
+
 OK, WARMUP, DEGENERATE = 0, 1, 2
 
 
@@ -274,10 +304,18 @@ class CutoffOracle:
     def reset(self):
         self.history = []
         self.step = 0
+        self.last_draws_sec = None       # predictive draws of the last decision, seconds, [S, N]
 
-    def push(self, runtimes_sec):
+    def push(self, runtimes_sec, censored=None):
+        """obs <- obs U r_w.  `censored` marks workers whose run-time was not observed (Section 4.2)."""
         x = np.asarray(runtimes_sec, dtype=np.float32)
-        assert x.shape == (self.N,) and np.all(np.isfinite(x)) and np.all(x > 0)
+        assert x.shape == (self.N,)
+        if censored is not None and np.any(censored):
+            assert self.last_draws_sec is not None, "imputation needs the predictive draws of this step"
+            x64, _ = impute_censored(np.where(np.asarray(censored).astype(bool), 0.0, x), censored,
+                                     self.last_draws_sec, self.seed, self.step)
+            x = x64.astype(np.float32)
+        assert np.all(np.isfinite(x)) and np.all(x > 0)
         self.history.append(x.copy())
 
     def scale(self) -> float:
@@ -297,7 +335,9 @@ class CutoffOracle:
         s = self.scale()
         rows = [self.samples(np.arange(k0, min(k0 + self.chunk, self.S)))   # rows are independent:
                 for k0 in range(0, self.S, self.chunk)]                     # chunking only bounds memory
-        expected = s * expected_order_statistics(np.concatenate(rows, axis=0))
+        draws = np.concatenate(rows, axis=0)
+        self.last_draws_sec = s * draws
+        expected = s * expected_order_statistics(draws)
         omega = throughput(expected)
         c, degenerate = argmax_cutoff(omega)
         self.step += 1

@@ -486,3 +486,61 @@ def test_noise_streams_feed_the_documented_stages():
             + math.exp(0.5 * float(w["b4"][n])) * O.normals(seed, step, O.STREAM_EMISSION, k, n))
     assert O.STREAM_TRANSITION == 0x100 and O.STREAM_EMISSION == 0x200
     assert np.allclose(x, want, rtol=0, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------
+# Censored run-times (Section 4.2)
+# ----------------------------------------------------------------------------
+def test_imputation_draws_from_the_left_truncated_predictive():
+    # every worker's predictive distribution is N(1.0, 0.2^2); censoring at 1.1 s
+    rng = np.random.default_rng(5)
+    S, N = 4000, 600
+    draws = rng.normal(1.0, 0.2, size=(S, N))
+    observed = np.full(N, 0.9)
+    observed[0] = 1.1                                  # the slowest worker that finished
+    censored = np.zeros(N, dtype=bool)
+    censored[100:] = True
+    x, threshold = O.impute_censored(observed, censored, draws, seed=77, step=3)
+    assert threshold == 1.1
+    assert np.array_equal(x[:100], observed[:100])     # what was observed is kept
+    assert np.all(x[100:] > threshold)
+    a = (threshold - 1.0) / 0.2
+    assert stats.kstest(x[100:], stats.truncnorm(a, np.inf, loc=1.0, scale=0.2).cdf).pvalue > 1e-3
+    assert abs(x[100:].mean() - stats.truncnorm(a, np.inf, loc=1.0, scale=0.2).mean()) < 4.5 * 0.12 / math.sqrt(500)
+    # each replacement is one of that worker's own predictive draws
+    assert all(x[j] in draws[:, j] for j in range(100, 130))
+    # same inputs, same result; another step number starts the scans elsewhere
+    x2, _ = O.impute_censored(observed, censored, draws, seed=77, step=3)
+    x3, _ = O.impute_censored(observed, censored, draws, seed=77, step=4)
+    assert np.array_equal(x, x2) and not np.array_equal(x, x3)
+
+
+def test_imputation_scan_order_and_fallback():
+    draws = np.array([[1.0, 5.0], [3.0, 5.0], [2.0, 5.0], [4.0, 0.5]])      # 4 draws, 2 workers
+    start = int(O.philox4x32_10(0, 0, O.STREAM_IMPUTE, 9, 21, 0)[0]) % 4
+    x, thr = O.impute_censored([0.0, 1.5], [True, False], draws, seed=21, step=9)
+    want = [v for v in np.roll(draws[:, 0], -start) if v > 1.5][0]          # first draw above 1.5 s from the start
+    assert thr == 1.5 and x[0] == want and x[1] == 1.5
+    # nothing above the threshold: the threshold itself
+    x, thr = O.impute_censored([0.0, 9.0], [True, False], draws, seed=21, step=9)
+    assert x[0] == 9.0
+    # no censoring: untouched
+    x, thr = O.impute_censored([0.7, 0.8], [False, False], draws, seed=21, step=9)
+    assert thr is None and list(x) == [0.7, 0.8]
+
+
+def test_oracle_push_with_censoring_uses_the_last_decision():
+    orc = _driven_oracle("tiny", 256)
+    code, c, e, omega = orc.predict()
+    wl = inputs.WORKLOADS["tiny"]
+    observed = inputs.workload_trace(wl, 21)[20]
+    order = np.argsort(observed)
+    censored = np.zeros(wl.N, dtype=bool)
+    censored[order[c:]] = True                         # the workers beyond the cutoff were killed
+    if c == wl.N:
+        censored[order[-2:]] = True
+    orc.push(observed, censored)
+    pushed = orc.history[-1]
+    assert np.array_equal(pushed[~censored], observed[~censored])
+    assert np.all(pushed[censored] >= observed[~censored].max())
+    assert orc.predict()[0] == O.OK
