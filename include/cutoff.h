@@ -114,9 +114,15 @@ int cutoff_load_weights(cutoff_ctx* ctx, const void* blob, size_t nbytes);
  * runtimes_sec: N floats, seconds, each finite and > 0; host memory if on_device == 0, device
  * memory on the context's device otherwise (then the check runs on the GPU and a bad value is
  * reported by this call after a stream synchronisation).
- * censored: must be NULL (imputation of censored run-times, Section 4.2, is not built):
- * non-NULL returns UNSUPPORTED.
- * The first lag+1 pushes fix the normaliser.  Errors: BAD_ARG, BAD_VALUE, UNSUPPORTED, CUDA. */
+ * censored: NULL, or N bytes in the same memory space as runtimes_sec; a non-zero byte marks a worker
+ * that was killed at the cutoff, whose run-time is therefore unknown and whose entry of runtimes_sec
+ * is ignored (Section 4.2).  Each such worker gets a draw from its own predictive distribution of this
+ * step, left-truncated at the largest observed run-time: the first of the S predictive draws of the
+ * last decision that exceeds it, scanning cyclically from a pseudo-random start; the threshold itself
+ * if none does.  Needs a completed decision since the last push (STATE otherwise), made in a single
+ * pass by a context that draws all samples of the decision (UNSUPPORTED otherwise), and at least one
+ * worker that finished.  Each decision's draws serve one censored push.
+ * The first lag+1 pushes fix the normaliser.  Errors: BAD_ARG, BAD_VALUE, STATE, UNSUPPORTED, CUDA. */
 int cutoff_push(cutoff_ctx* ctx, const float* runtimes_sec, int on_device, const uint8_t* censored);
 
 /* As cutoff_push with a device pointer, but only enqueues: no synchronisation, no error report
@@ -200,6 +206,9 @@ int cutoff_set_option(cutoff_ctx* ctx, const char* name, int64_t value);
 int cutoff_debug_normals(int device, uint64_t seed, uint32_t step, uint32_t stream, int64_t k0,
                          int64_t count, int32_t n_elems, float* normals_out, uint32_t* words_out);
 int cutoff_debug_samples(cutoff_ctx* ctx, int64_t k0, int64_t count, float* x_out);
+/* cutoff_debug_window: the observation window as the encoder will see it, oldest vector first, in
+ * seconds (window_out, host, (lag+1)*N floats); imputed entries included.  WARMUP before lag+1 pushes. */
+int cutoff_debug_window(cutoff_ctx* ctx, float* window_out);
 int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n,
                       float* keys_out, int32_t* perm_out);
 

@@ -30,7 +30,8 @@ EXPORTS = (
     "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
-    "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_sort", "cutoff_sorted_row_sums_static",
+    "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
+    "cutoff_sorted_row_sums_static",
 )
 
 
@@ -88,6 +89,7 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_debug_normals": (C.c_int, [C.c_int, C.c_uint64, C.c_uint32, C.c_uint32, C.c_int64, C.c_int64,
                                            C.c_int32, vp, vp]),
         "cutoff_debug_samples": (C.c_int, [vp, C.c_int64, C.c_int64, vp]),
+        "cutoff_debug_window": (C.c_int, [vp, vp]),
         "cutoff_debug_sort": (C.c_int, [vp, vp, C.c_int64, C.c_int32, vp, vp]),
         "cutoff_sorted_row_sums_static": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
     }
@@ -159,16 +161,27 @@ class Cutoff:
         blob = weights if isinstance(weights, (bytes, bytearray)) else pack_weights(weights, self.N, self.D, self.H)
         self._check(self._lib.cutoff_load_weights(self._h, blob, len(blob)), "cutoff_load_weights")
 
-    def push(self, runtimes_sec) -> int:
-        """Host numpy array (fp32, N) or torch CUDA tensor."""
+    def push(self, runtimes_sec, censored=None) -> int:
+        """Host numpy array (fp32, N) or torch CUDA tensor; `censored` (same kind, N bytes / bools) marks killed workers."""
         if isinstance(runtimes_sec, np.ndarray):
             a = np.ascontiguousarray(runtimes_sec, dtype=np.float32)
             if a.shape != (self.N,):
                 raise ValueError("expected N run-times")
-            return self._check(self._lib.cutoff_push(self._h, a.ctypes.data, 0, None), "cutoff_push")
+            mask = None
+            if censored is not None:
+                mask = np.ascontiguousarray(np.asarray(censored).astype(np.uint8))
+                if mask.shape != (self.N,):
+                    raise ValueError("expected N censoring flags")
+            return self._check(self._lib.cutoff_push(self._h, a.ctypes.data, 0, mask.ctypes.data if mask is not None else None),
+                               "cutoff_push")
         if tuple(runtimes_sec.shape) != (self.N,) or not runtimes_sec.is_cuda or not runtimes_sec.is_contiguous():
             raise ValueError("expected a contiguous CUDA tensor of N fp32 run-times")
-        return self._check(self._lib.cutoff_push(self._h, runtimes_sec.data_ptr(), 1, None), "cutoff_push")
+        mask_ptr = None
+        if censored is not None:
+            if tuple(censored.shape) != (self.N,) or not censored.is_cuda or censored.element_size() != 1:
+                raise ValueError("expected a CUDA tensor of N one-byte censoring flags")
+            mask_ptr = censored.data_ptr()
+        return self._check(self._lib.cutoff_push(self._h, runtimes_sec.data_ptr(), 1, mask_ptr), "cutoff_push")
 
     def push_async(self, runtimes_sec_device) -> int:
         return self._check(self._lib.cutoff_push_async(self._h, runtimes_sec_device.data_ptr()), "cutoff_push_async")
@@ -249,6 +262,13 @@ class Cutoff:
         if rc == WARMUP:
             raise CutoffError(ERR_STATE, "cutoff_debug_samples", "fewer than lag+1 observations")
         return x
+
+    def debug_window(self) -> np.ndarray:
+        w = np.empty((self.lag + 1, self.N), dtype=np.float32)
+        rc = self._check(self._lib.cutoff_debug_window(self._h, w.ctypes.data), "cutoff_debug_window")
+        if rc == WARMUP:
+            raise CutoffError(ERR_STATE, "cutoff_debug_window", "fewer than lag+1 observations")
+        return w
 
     def debug_sort(self, rows: np.ndarray):
         r = np.ascontiguousarray(rows, dtype=np.float32)

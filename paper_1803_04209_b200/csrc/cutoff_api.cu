@@ -48,6 +48,9 @@ struct cutoff_ctx {
 
     float* d_ring = nullptr;        // [W][N]
     float* d_stage = nullptr;       // [N] landing buffer for host pushes
+    uint8_t* d_mask = nullptr;      // [N] censoring mask of the push in progress
+    uint8_t* h_mask = nullptr;      // pinned [N]
+    bool draws_valid = false;       // d_x holds every predictive draw of the last decision (needed for imputation)
     DevState* d_state = nullptr;
     float* d_proj = nullptr;        // [2][W][H]
     float* d_hlr = nullptr;         // [2][W][H]
@@ -115,7 +118,8 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
-    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_chain_image); cudaFree(c->d_ring); cudaFree(c->d_stage);
+    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
+    if (c->h_mask) cudaFreeHost(c->h_mask); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
     cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
     if (c->h_stage) cudaFreeHost(c->h_stage);
@@ -457,6 +461,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_mask, c->N));
+    CREATE_CHECK(cudaMallocHost(&c->h_mask, c->N));
     CREATE_CHECK(cudaMalloc(&c->d_state, sizeof(DevState)));
     CREATE_CHECK(cudaMalloc(&c->d_proj, sizeof(float) * 2 * c->W * c->H));
     CREATE_CHECK(cudaMalloc(&c->d_hlr, sizeof(float) * 2 * c->W * c->H));
@@ -603,10 +609,50 @@ int cutoff_push_async(cutoff_ctx* c, const float* runtimes_sec_device) {
     return push_common(c, runtimes_sec_device);
 }
 
+// Push with a censoring mask: land run-times and mask on the device, replace the censored entries by
+// draws from the truncated predictive distribution of the last decision, then push as usual.
+static int push_censored(cutoff_ctx* c, const float* runtimes_sec, int on_device, const uint8_t* censored) {
+    if (!c->draws_valid) return CUTOFF_ERR_STATE;          // no decision yet whose draws could be used
+    if (c->cfg.sample_offset != 0 || (c->cfg.total_samples > 0 && c->cfg.total_samples != c->S))
+        return CUTOFF_ERR_UNSUPPORTED;                      // a context that holds only part of the draws
+    const cudaMemcpyKind kind = on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice;
+    if (!on_device) {
+        int finished = 0;
+        for (int j = 0; j < c->N; ++j) {
+            if (censored[j]) continue;
+            if (!(runtimes_sec[j] > 0.0f) || !std::isfinite(runtimes_sec[j])) return CUTOFF_ERR_BAD_VALUE;
+            ++finished;
+        }
+        if (finished == 0) return CUTOFF_ERR_BAD_ARG;
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));     // the landing buffers may still be in use
+        for (int j = 0; j < c->N; ++j) c->h_stage[j] = censored[j] ? 1.0f : runtimes_sec[j];
+        std::memcpy(c->h_mask, censored, c->N);
+        CU_CHECK(c, cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, kind, c->stream));
+        CU_CHECK(c, cudaMemcpyAsync(c->d_mask, c->h_mask, c->N, kind, c->stream));
+    } else {
+        CU_CHECK(c, cudaMemcpyAsync(c->d_stage, runtimes_sec, sizeof(float) * c->N, kind, c->stream));
+        CU_CHECK(c, cudaMemcpyAsync(c->d_mask, censored, c->N, kind, c->stream));
+    }
+    const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    k_impute<<<1, kImputeThreads, 0, c->stream>>>(c->d_stage, c->d_mask, c->d_x, c->ldx, c->S, c->N, c->d_state, key);
+    c->launches += 1;
+    c->draws_valid = false;                                 // one step's draws serve one push
+    int rc = push_common(c, c->d_stage);
+    if (rc) return rc;
+    CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    if (c->h_state->error_flags & kErrBadValue) {
+        c->pushes = c->h_state->push_count;
+        CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
+        return CUTOFF_ERR_BAD_VALUE;
+    }
+    return CUTOFF_OK;
+}
+
 int cutoff_push(cutoff_ctx* c, const float* runtimes_sec, int on_device, const uint8_t* censored) {
     if (!c || !runtimes_sec) return CUTOFF_ERR_BAD_ARG;
-    if (censored) return CUTOFF_ERR_UNSUPPORTED;
     CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (censored) return push_censored(c, runtimes_sec, on_device, censored);
     if (!on_device) {
         for (int j = 0; j < c->N; ++j)
             if (!(runtimes_sec[j] > 0.0f) || !std::isfinite(runtimes_sec[j])) return CUTOFF_ERR_BAD_VALUE;
@@ -665,6 +711,7 @@ int cutoff_fetch(cutoff_ctx* c, int32_t* c_out) {
     if (rc) return rc;
     c->have_result = true;
     c->decided_once = true;
+    c->draws_valid = c->n_chunks == 1;
     *c_out = c->h_state->c_star;
     return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
 }
@@ -727,6 +774,7 @@ int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     c->launches += c->graph_kernels;
     c->pushes += 1;
+    c->draws_valid = c->n_chunks == 1;
     if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
     c->have_result = true;
     *c_out = c->h_state->c_star;
@@ -779,6 +827,7 @@ int cutoff_reset(cutoff_ctx* c) {
     c->pushes = 0;
     c->pending = false;
     c->have_result = false;
+    c->draws_valid = false;
     return CUTOFF_OK;
 }
 
@@ -908,6 +957,7 @@ int cutoff_debug_samples(cutoff_ctx* c, int64_t k0, int64_t count, float* x_out)
     if (!c->weights_loaded || c->pending) return CUTOFF_ERR_STATE;
     if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
     CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    c->draws_valid = false;                                 // the sample matrix is about to be overwritten
     launch_encoder(c);
     for (int64_t done = 0; done < count; done += c->chunk_rows) {
         const int n = static_cast<int>(count - done < c->chunk_rows ? count - done : c->chunk_rows);
@@ -919,6 +969,20 @@ int cutoff_debug_samples(cutoff_ctx* c, int64_t k0, int64_t count, float* x_out)
         CU_CHECK(c, cudaStreamSynchronize(c->stream));
     }
     CU_CHECK(c, cudaGetLastError());
+    return CUTOFF_OK;
+}
+
+int cutoff_debug_window(cutoff_ctx* c, float* window_out) {
+    if (!c || !window_out) return CUTOFF_ERR_BAD_ARG;
+    if (c->pending) return CUTOFF_ERR_STATE;
+    if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    for (int t = 0; t < c->W; ++t) {                       // position t (0 = oldest) sits in slot (pushes + t) mod W
+        const size_t slot = (static_cast<size_t>(c->pushes) + t) % c->W;
+        CU_CHECK(c, cudaMemcpy(window_out + static_cast<size_t>(t) * c->N, c->d_ring + slot * c->N, sizeof(float) * c->N,
+                               cudaMemcpyDeviceToHost));
+    }
     return CUTOFF_OK;
 }
 

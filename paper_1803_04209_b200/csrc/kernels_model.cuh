@@ -52,6 +52,64 @@ __global__ void __launch_bounds__(kPushThreads) k_push(const float* __restrict__
 }
 
 // ---------------------------------------------------------------------------------------------
+// Censored run-times (Section 4.2): a worker that was killed at the cutoff gets a draw from its own
+// predictive distribution of this step, left-truncated at the cutoff time (the largest run-time
+// that was observed).  The predictive distribution is the Monte-Carlo one: column j of the sample
+// matrix of the last decision.  The draws are iid, so the first one above the threshold, scanning
+// cyclically from a start that does not depend on their values (Philox word 0 of counter
+// (worker, 0, 0x300, decision number) modulo S), is an exact draw from the truncated distribution;
+// if there is none the threshold itself is used.  One CTA; a warp per censored worker.
+// ---------------------------------------------------------------------------------------------
+constexpr int kImputeThreads = 1024;
+constexpr uint32_t kStreamImpute = 0x300u;
+
+__global__ void __launch_bounds__(kImputeThreads) k_impute(float* __restrict__ stage, const uint8_t* __restrict__ censored,
+                                                            const float* __restrict__ x, int ldx, int S, int N,
+                                                            const DevState* __restrict__ st, NoiseKey key) {
+    __shared__ float red[kImputeThreads / 32];
+    __shared__ float s_threshold;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float m = -INFINITY;
+    for (int j = threadIdx.x; j < N; j += kImputeThreads)
+        if (!censored[j]) m = fmaxf(m, stage[j]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if (lane == 0) red[warp] = m;
+    __syncthreads();
+    if (warp == 0) {
+        m = red[lane];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+        if (lane == 0) s_threshold = m;
+    }
+    __syncthreads();
+    const float threshold = s_threshold;          // -inf if nobody finished: the push that follows rejects the vector
+    const float scale = st->scale;
+    const uint32_t step = st->step;
+    for (int j = warp; j < N; j += kImputeThreads / 32) {
+        if (!censored[j]) continue;
+        const uint32_t start = philox4x32_10(static_cast<uint32_t>(j), 0u, kStreamImpute, step, key.seed_lo, key.seed_hi).x %
+                               static_cast<uint32_t>(S);
+        float value = threshold;
+        for (int base = 0; base < S; base += 32) {
+            const int i = base + lane;
+            float v = -INFINITY;
+            if (i < S) {
+                uint32_t k = start + static_cast<uint32_t>(i);
+                if (k >= static_cast<uint32_t>(S)) k -= static_cast<uint32_t>(S);
+                v = x[static_cast<size_t>(k) * ldx + j] * scale;
+            }
+            const uint32_t hit = __ballot_sync(0xffffffffu, v > threshold);
+            if (hit) {
+                value = __shfl_sync(0xffffffffu, v, __ffs(hit) - 1);
+                break;
+            }
+        }
+        if (lane == 0) stage[j] = value;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Encoder, part 1: input projections of both RNNs for every window position,
 //   P[dir][t][i] = sum_j Wx_dir[i][j] * xhat_t[j] + b_dir[i],   xhat_t = x_t / s.
 // One warp per hidden unit i; the weight row is read once for all window positions.

@@ -332,11 +332,73 @@ def test_errors_are_codes_not_crashes():
     assert gpu.predict() == (binding.WARMUP, wl.N)
     gpu.push(good)
     assert gpu.predict()[0] == binding.OK
-    import ctypes as C
-    flag = (C.c_uint8 * wl.N)()
-    assert gpu._lib.cutoff_push(gpu._h, good.ctypes.data, 0, flag) == binding.ERR_UNSUPPORTED
     with pytest.raises(binding.CutoffError) as e:
         gpu.fetch()                                     # nothing enqueued
+    assert e.value.code == binding.ERR_STATE
+
+
+def _censor_beyond_cutoff(observed, c):
+    order = np.argsort(observed, kind="stable")
+    censored = np.zeros(observed.shape[0], dtype=bool)
+    censored[order[min(c, observed.shape[0] - 3):]] = True          # at least the three slowest are killed
+    return censored
+
+
+@pytest.mark.parametrize("name,S", [("n128", 2048), ("n1024", 1024)])
+def test_censored_push_imputes_from_the_truncated_predictive(name, S):
+    import torch
+    wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 5)
+    tol = TOL_X[prec]
+    observed = inputs.workload_trace(wl, wl.window + 6)[-1]
+    with pytest.raises(binding.CutoffError) as e:                   # no decision yet: nothing to draw from
+        gpu.push(observed, np.ones(wl.N, dtype=bool))
+    assert e.value.code == binding.ERR_STATE
+    x_gpu = gpu.debug_samples(0, S).astype(np.float64) * orc.scale()   # the draws the decision is about to make
+    code_o, c_o, _, _ = orc.predict()
+    code_g, c_g = gpu.predict()
+    assert code_g == code_o == binding.OK
+    censored = _censor_beyond_cutoff(observed, c_o)
+    with pytest.raises(binding.CutoffError) as e:                   # nobody finished
+        gpu.push(observed, np.ones(wl.N, dtype=bool))
+    assert e.value.code == binding.ERR_BAD_ARG
+    junk = observed.copy()
+    junk[censored] = np.nan                                         # censored entries are ignored
+    gpu.push(junk, censored)
+    orc.push(observed, censored)
+    got = gpu.debug_window()[-1].astype(np.float64)
+    want = orc.history[-1].astype(np.float64)
+    threshold = float(observed[~censored].max())
+    assert np.array_equal(got[~censored], observed[~censored].astype(np.float64))
+    assert np.all(got[censored] >= threshold)
+    # every replacement is the first of the worker's own draws above the threshold, in the oracle's scan order
+    draws = orc.last_draws_sec
+    checked = 0
+    for j in np.flatnonzero(censored):
+        start = int(O.philox4x32_10(int(j), 0, O.STREAM_IMPUTE, orc.step, SEED & 0xFFFFFFFF, SEED >> 32)[0]) % S
+        col = np.roll(draws[:, j], -start)
+        hits = np.flatnonzero(col > threshold)
+        upto = col[: hits[0] + 1] if hits.size else col
+        if np.any(np.abs(upto - threshold) <= 2 * tol * threshold):
+            continue                                                # a draw too close to the threshold to call
+        checked += 1
+        assert abs(got[j] - want[j]) <= tol * max(abs(want[j]), threshold)
+        k_star = (start + hits[0]) % S if hits.size else None
+        if k_star is not None:
+            assert abs(got[j] - x_gpu[k_star, j]) <= 1e-6 * abs(got[j])     # it is the GPU's own draw
+    assert checked >= 0.8 * censored.sum()
+    # the imputed window feeds the next decision
+    assert_decision_close(gpu, orc.predict(), wl.N)
+    # device pointers take the same path
+    _, gpu2, _, _ = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 5)
+    gpu2.predict()
+    gpu2.push(torch.from_numpy(np.where(censored, 1.0, observed).astype(np.float32)).cuda(),
+              torch.from_numpy(censored.astype(np.uint8)).cuda())
+    assert np.array_equal(gpu2.debug_window()[-1], got.astype(np.float32))
+    # a push without censored workers is an ordinary push; a second censored push needs a new decision
+    gpu2.predict()
+    assert gpu2.push(observed, np.zeros(wl.N, dtype=bool)) == binding.OK
+    with pytest.raises(binding.CutoffError) as e:
+        gpu2.push(observed, censored)
     assert e.value.code == binding.ERR_STATE
 
 
