@@ -43,6 +43,7 @@ struct cutoff_ctx {
 
     float* d_blob = nullptr;        // tensors as loaded
     float* d_WT = nullptr;          // transposed copies WzT, W1T, W3T: 3 x [D][H]
+    float* d_WhR = nullptr;         // recurrence matrices regrouped per thread for k_enc_rnn_resident: 2 x H x H
     ModelDev m{};
     bool weights_loaded = false;
 
@@ -118,7 +119,7 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
-    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
+    cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_WhR); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
     if (c->h_mask) cudaFreeHost(c->h_mask); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
     cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
@@ -299,7 +300,7 @@ void launch_rnn_resident(cutoff_ctx* c) {
         attr_set = true;
     }
     const size_t smem = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float);
-    k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_proj, c->d_hlr);
+    k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_WhR, c->d_proj, c->d_hlr);
 }
 
 void launch_encoder(cutoff_ctx* c) {
@@ -458,6 +459,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
     CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
     CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 3 * c->H * c->D));
+    CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
@@ -541,6 +543,20 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     }
     CU_CHECK(c, cudaMemcpy(c->d_WT, wT.data(), wT.size() * sizeof(float), cudaMemcpyHostToDevice));
 
+    {
+        // recurrence matrices regrouped per thread of k_enc_rnn_resident: [dir][j4][thread = 4*i + q][4]
+        const size_t HQ = H / 4, T = 4 * H;
+        std::vector<float> whr(2 * H * H);
+        const size_t src_off[2] = {off[1], off[5]};                   // Whf, Whb: each [H][H]
+        for (int dir = 0; dir < 2; ++dir) {
+            const float* w = host.data() + src_off[dir];
+            for (size_t i = 0; i < H; ++i)
+                for (size_t q = 0; q < 4; ++q)
+                    for (size_t j = 0; j < HQ; ++j)
+                        whr[dir * H * H + ((j / 4) * T + (4 * i + q)) * 4 + (j % 4)] = w[i * H + q * HQ + j];
+        }
+        CU_CHECK(c, cudaMemcpy(c->d_WhR, whr.data(), whr.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
     if (c->chain_tc) {
         // Operand tiles of the tensor-core chain as they will sit in shared memory: tf32 (nearest, ties
         // away), K-major rows of 32 values, 16-byte chunks XOR-swizzled with the row index modulo 8.

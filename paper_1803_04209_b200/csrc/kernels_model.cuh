@@ -217,7 +217,8 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
 // double-buffered in shared memory, so a step costs one __syncthreads.
 // ---------------------------------------------------------------------------------------------
 template <int HQ>   // HQ = H / 4
-__global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const float* __restrict__ proj,
+__global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const float* __restrict__ wh_threads,
+                                                              const float* __restrict__ proj,
                                                               float* __restrict__ hlr /*[2][W][H]*/) {
     constexpr int H = 4 * HQ, T = 16 * HQ, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ, PAD = HQ + 4;
     extern __shared__ __align__(16) float sm_rr[];
@@ -226,18 +227,19 @@ __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const 
     float* swh = sproj + m.W * H;                 // [SQ/4][T][4]
     const int dir = blockIdx.x;
     const int t = threadIdx.x, i = t >> 2, q = t & 3;
-    const float* Wh = (dir ? m.Whb : m.Whf) + static_cast<size_t>(i) * H + q * HQ;
+    // wh_threads holds both recurrence matrices regrouped per thread, [dir][j4][thread][4]: the j4-th group of
+    // four weights of thread (i, q) is Wh[i][q*HQ + 4*j4 ..], so that consecutive threads read consecutive 16 bytes
+    const float4* Wh = reinterpret_cast<const float4*>(wh_threads) + static_cast<size_t>(dir) * (HQ / 4) * T;
     const float* init = dir ? m.b0 : m.a0;
     float w[RQ];
 #pragma unroll
     for (int j4 = 0; j4 < RQ / 4; ++j4) {
-        const float4 v = *reinterpret_cast<const float4*>(Wh + 4 * j4);
+        const float4 v = Wh[static_cast<size_t>(j4) * T + t];
         w[4 * j4 + 0] = v.x; w[4 * j4 + 1] = v.y; w[4 * j4 + 2] = v.z; w[4 * j4 + 3] = v.w;
     }
 #pragma unroll
     for (int j4 = 0; j4 < SQ / 4; ++j4)
-        *reinterpret_cast<float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4) =
-            *reinterpret_cast<const float4*>(Wh + RQ + 4 * j4);
+        *reinterpret_cast<float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4) = Wh[static_cast<size_t>(RQ / 4 + j4) * T + t];
     for (int idx = t; idx < m.W * H; idx += T) sproj[idx] = proj[static_cast<size_t>(dir) * m.W * H + idx];
     if (t < H) state[(t / HQ) * PAD + (t % HQ)] = init[t];
     __syncthreads();
