@@ -154,6 +154,12 @@ int cutoff_step(cutoff_ctx* ctx, const float* runtimes_sec, int32_t* c_out);
  * Errors: STATE if no decision has completed, CUDA. */
 int cutoff_get_stats(cutoff_ctx* ctx, float* exp_order_stats_sec, float* omega_per_sec);
 
+/* Spread of each order statistic over the samples of the last decision: the standard deviation of
+ * x~_(j), in seconds (std_sec, host, N floats) -- the +-2 sigma bands the paper draws around the predicted
+ * order statistics (Fig. 3).  Computed only by decisions made after
+ * cutoff_set_option(ctx, "order_stat_std", 1) (the sort then also accumulates squares); STATE otherwise. */
+int cutoff_get_order_stat_std(cutoff_ctx* ctx, float* std_sec);
+
 /* Sum over this context's samples of the sorted, normalised run-times of the last decision
  * (host, N doubles): the quantity several contexts add up when they share one decision.
  * cutoff_decide_from_sums then finishes a decision from such a total: sums (host, N doubles)
@@ -186,8 +192,11 @@ int cutoff_get_timing(cutoff_ctx* ctx, float* ms, int cap);
 const char* cutoff_stage_name(int i);
 int64_t cutoff_launch_count(cutoff_ctx* ctx);
 
-/* Tuning knobs, by name.  "pass_rows": samples that go through sampling and sorting per pass
- * (>= 1024; clipped to S and to the allocated pass buffers).  Errors: BAD_ARG, STATE. */
+/* Options, by name.  "pass_rows": samples that go through sampling and sorting per pass (>= 1024;
+ * clipped to S and to the allocated pass buffers).  "order_stat_std": 1 = also compute the spread
+ * of each order statistic (see cutoff_get_order_stat_std), 0 = do not (default); not available to a
+ * context that holds only part of a decision's samples (UNSUPPORTED), nor once a graph has been
+ * captured (STATE).  Errors: BAD_ARG, STATE, UNSUPPORTED. */
 int cutoff_set_option(cutoff_ctx* ctx, const char* name, int64_t value);
 
 /* ---- test hooks ----------------------------------------------------------------------------

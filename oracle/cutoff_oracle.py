@@ -231,6 +231,11 @@ def expected_order_statistics(x: np.ndarray) -> np.ndarray:
     return np.sort(x, axis=1, kind="stable").mean(axis=0)
 
 
+def order_statistic_std(x: np.ndarray) -> np.ndarray:
+    """Standard deviation over the samples of each sorted position (the +-2 sigma bands of Fig. 3)."""
+    return np.sort(x, axis=1, kind="stable").std(axis=0)
+
+
 def throughput(expected_sorted: np.ndarray) -> np.ndarray:
     """Omega(c) = c / E[x~_(c)] for c = 1..N; minus infinity where the expectation is not positive."""
     e = np.asarray(expected_sorted, dtype=np.float64)
@@ -337,6 +342,7 @@ class CutoffOracle:
                 for k0 in range(0, self.S, self.chunk)]                     # chunking only bounds memory
         draws = np.concatenate(rows, axis=0)
         self.last_draws_sec = s * draws
+        self.last_std_sec = s * order_statistic_std(draws)
         expected = s * expected_order_statistics(draws)
         omega = throughput(expected)
         c, degenerate = argmax_cutoff(omega)

@@ -27,7 +27,7 @@ BLOB_MAGIC = 0x31465443
 EXPORTS = (
     "cutoff_create", "cutoff_destroy", "cutoff_load_weights", "cutoff_push", "cutoff_push_async",
     "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_step", "cutoff_get_stats",
-    "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
+    "cutoff_get_order_stat_std", "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
     "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
@@ -74,6 +74,7 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_fetch": (C.c_int, [vp, i32p]),
         "cutoff_step": (C.c_int, [vp, vp, i32p]),
         "cutoff_get_stats": (C.c_int, [vp, vp, vp]),
+        "cutoff_get_order_stat_std": (C.c_int, [vp, vp]),
         "cutoff_get_partial_sums": (C.c_int, [vp, vp]),
         "cutoff_decide_from_sums": (C.c_int, [vp, vp, i32p]),
         "cutoff_reset": (C.c_int, [vp]),
@@ -215,6 +216,12 @@ class Cutoff:
         om = np.empty(self.N, dtype=np.float32)
         self._check(self._lib.cutoff_get_stats(self._h, e.ctypes.data, om.ctypes.data), "cutoff_get_stats")
         return e, om
+
+    def get_order_stat_std(self) -> np.ndarray:
+        """Standard deviation of each order statistic over the samples (seconds); needs option order_stat_std."""
+        sd = np.empty(self.N, dtype=np.float32)
+        self._check(self._lib.cutoff_get_order_stat_std(self._h, sd.ctypes.data), "cutoff_get_order_stat_std")
+        return sd
 
     def get_partial_sums(self) -> np.ndarray:
         s = np.empty(self.N, dtype=np.float64)

@@ -57,7 +57,10 @@ struct cutoff_ctx {
     float* d_hlr = nullptr;         // [2][W][H]
     float* d_v = nullptr;           // [chunk_rows][H]
     float* d_x = nullptr;           // [chunk_rows][ldx]
-    float* d_partial = nullptr;     // [n_chunks * sort_grid][N]
+    float* d_partial = nullptr;     // [n_chunks * sort_grid][N]; a second block of kPartialRows rows holds sums of squares
+    float* d_std = nullptr;         // [N] spread of each order statistic (when asked for)
+    bool want_std = false;
+    bool have_std = false;
     double* d_sums = nullptr;       // [N]
     float* d_E = nullptr;           // [N]
     float* d_omega = nullptr;       // [N]
@@ -122,7 +125,7 @@ void free_all(cutoff_ctx* c) {
     cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_WhR); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
     if (c->h_mask) cudaFreeHost(c->h_mask); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
-    cudaFree(c->d_partial); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
+    cudaFree(c->d_partial); cudaFree(c->d_std); cudaFree(c->d_sums); cudaFree(c->d_E); cudaFree(c->d_omega);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->h_state) cudaFreeHost(c->h_state);
     if (c->owns_stream && c->stream) cudaStreamDestroy(c->stream);
@@ -151,15 +154,29 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
     c->sort_grid = want < cap ? want : cap;
 }
 
-template <int E>
-void launch_sort_warp(cutoff_ctx* c, int count, float* partial) {
+template <int E, bool SQ>
+void launch_sort_warp_sq(cutoff_ctx* c, int count, float* partial) {
     static bool attr_set = false;
     const size_t smem = sort_tma_smem_bytes<E>(c->ldx);
     if (!attr_set) {
-        cudaFuncSetAttribute(k_sort_sum_tma<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
+        cudaFuncSetAttribute(k_sort_sum_tma<E, SQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
         attr_set = true;
     }
-    k_sort_sum_tma<E><<<c->sort_grid, kSortWarps * 32, smem, c->stream>>>(c->d_x, c->ldx, c->N, count, partial, c->d_state);
+    k_sort_sum_tma<E, SQ><<<c->sort_grid, kSortWarps * 32, smem, c->stream>>>(
+        c->d_x, c->ldx, c->N, count, partial, partial + static_cast<size_t>(kPartialRows) * c->N, c->d_state);
+}
+
+template <int E>
+void launch_sort_warp(cutoff_ctx* c, int count, float* partial) {
+    if (c->want_std) launch_sort_warp_sq<E, true>(c, count, partial);
+    else launch_sort_warp_sq<E, false>(c, count, partial);
+}
+
+template <int WPR>
+void launch_sort_cta(cutoff_ctx* c, int count, float* partial) {
+    float* partial_sq = partial + static_cast<size_t>(kPartialRows) * c->N;
+    if (c->want_std) k_sort_sum_cta<WPR, true><<<c->sort_grid, WPR * 32, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial, partial_sq);
+    else k_sort_sum_cta<WPR, false><<<c->sort_grid, WPR * 32, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial, partial_sq);
 }
 
 int launch_sort(cutoff_ctx* c, int count, float* partial) {
@@ -170,12 +187,8 @@ int launch_sort(cutoff_ctx* c, int count, float* partial) {
         case 256: launch_sort_warp<8>(c, count, partial); break;
         case 512: launch_sort_warp<16>(c, count, partial); break;
         case 1024: launch_sort_warp<32>(c, count, partial); break;
-        case 2048:
-            k_sort_sum_cta<2><<<c->sort_grid, 64, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
-            break;
-        case 4096:
-            k_sort_sum_cta<4><<<c->sort_grid, 128, 0, c->stream>>>(c->d_x, c->ldx, c->N, count, partial);
-            break;
+        case 2048: launch_sort_cta<2>(c, count, partial); break;
+        case 4096: launch_sort_cta<4>(c, count, partial); break;
         default: return CUTOFF_ERR_UNSUPPORTED;
     }
     c->launches += 1;
@@ -352,7 +365,10 @@ int enqueue_decision(cutoff_ctx* c) {
     const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
     k_colsum_decide<<<ceil_div(c->N, 32), kColsumThreads, 0, c->stream>>>(c->d_partial, c->n_chunks * c->sort_grid, c->N,
                                                                          c->d_sums, 1.0 / static_cast<double>(total),
-                                                                         c->d_state, c->d_E, c->d_omega);
+                                                                         c->d_state, c->d_E, c->d_omega,
+                                                                         c->want_std ? c->d_partial + static_cast<size_t>(kPartialRows) * c->N : nullptr,
+                                                                         c->d_std);
+    c->have_std = c->want_std;
     c->launches += 1;
     if (timed) cudaEventRecord(c->ev[5][0], c->stream);
     c->timed_chunks = timed ? c->n_chunks : 0;
@@ -470,7 +486,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_hlr, sizeof(float) * 2 * c->W * c->H));
     CREATE_CHECK(cudaMalloc(&c->d_v, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->H));
     CREATE_CHECK(cudaMalloc(&c->d_x, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
-    CREATE_CHECK(cudaMalloc(&c->d_partial, sizeof(float) * static_cast<size_t>(kPartialRows) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_partial, sizeof(float) * 2 * static_cast<size_t>(kPartialRows) * c->N));
+    CREATE_CHECK(cudaMalloc(&c->d_std, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_sums, sizeof(double) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_E, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_omega, sizeof(float) * c->N));
@@ -808,6 +825,15 @@ int cutoff_get_stats(cutoff_ctx* c, float* e_out, float* omega_out) {
     return CUTOFF_OK;
 }
 
+int cutoff_get_order_stat_std(cutoff_ctx* c, float* std_sec) {
+    if (!c || !std_sec) return CUTOFF_ERR_BAD_ARG;
+    if (!c->have_result || !c->have_std) return CUTOFF_ERR_STATE;
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    CU_CHECK(c, cudaMemcpyAsync(std_sec, c->d_std, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    return CUTOFF_OK;
+}
+
 int cutoff_get_partial_sums(cutoff_ctx* c, double* sums) {
     if (!c || !sums) return CUTOFF_ERR_BAD_ARG;
     if (!c->have_result) return CUTOFF_ERR_STATE;
@@ -905,6 +931,13 @@ int64_t cutoff_launch_count(cutoff_ctx* c) { return c ? c->launches : 0; }
 int cutoff_set_option(cutoff_ctx* c, const char* name, int64_t value) {
     if (!c || !name) return CUTOFF_ERR_BAD_ARG;
     if (c->pending) return CUTOFF_ERR_STATE;
+    if (std::strcmp(name, "order_stat_std") == 0) {
+        if (value != 0 && value != 1) return CUTOFF_ERR_BAD_ARG;
+        if (value && c->cfg.total_samples > 0 && c->cfg.total_samples != c->S) return CUTOFF_ERR_UNSUPPORTED;
+        if (c->graph_exec) return CUTOFF_ERR_STATE;                // the captured graph has the other sort kernel in it
+        c->want_std = value != 0;
+        return CUTOFF_OK;
+    }
     if (std::strcmp(name, "pass_rows") == 0) {
         if (value < 1024) return CUTOFF_ERR_BAD_ARG;
         plan_chunks(c, static_cast<int>(value));

@@ -247,9 +247,10 @@ inline size_t sort_tma_smem_bytes(int ldx) {
     return (rows > stage ? rows : stage) + 16 * kSortWarps + 16;
 }
 
-template <int E>
+template <int E, bool SQ>
 __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* __restrict__ x, int ldx, int N, int count,
-                                                                   float* __restrict__ partial, DevState* st) {
+                                                                   float* __restrict__ partial,
+                                                                   float* __restrict__ partial_sq, DevState* st) {
     using namespace cutoff::async;
     extern __shared__ __align__(16) float sm_sort[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -270,9 +271,11 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
     }
     __syncthreads();
 
-    float acc[E];
+    float acc[E], acc_sq[SQ ? E : 1];
 #pragma unroll
     for (int r = 0; r < E; ++r) acc[r] = 0.0f;
+#pragma unroll
+    for (int r = 0; r < (SQ ? E : 1); ++r) acc_sq[r] = 0.0f;
     const int stride = gridDim.x * kSortWarps;
     int row = blockIdx.x * kSortWarps + warp;
     if (row < count && lane == 0) {
@@ -312,6 +315,10 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
         warp_bitonic_sort<float, E>(v, lane);
 #pragma unroll
         for (int r = 0; r < E; ++r) acc[r] += v[r];
+        if (SQ) {
+#pragma unroll
+            for (int r = 0; r < E; ++r) acc_sq[SQ ? r : 0] = fmaf(v[r], v[r], acc_sq[SQ ? r : 0]);
+        }
     }
     (void)aborted;
     __syncthreads();                                   // all row buffers are dead: reuse them as the stage
@@ -325,20 +332,34 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
         for (int w = 0; w < kSortWarps; ++w) s += stage[w * 32 * E + j];
         partial[static_cast<size_t>(blockIdx.x) * N + j] = s;
     }
+    if (SQ) {                                          // the same reduction for the sums of squares
+        __syncthreads();
+#pragma unroll
+        for (int r = 0; r < E; ++r) stage[warp * 32 * E + lane * E + r] = acc_sq[SQ ? r : 0];
+        __syncthreads();
+        for (int j = threadIdx.x; j < N; j += kSortWarps * 32) {
+            float s = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kSortWarps; ++w) s += stage[w * 32 * E + j];
+            partial_sq[static_cast<size_t>(blockIdx.x) * N + j] = s;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
 // Sort + accumulate for wide rows (1024 < N <= 4096): a CTA of WPR = P/1024 warps per row, keys in
 // registers, running sums in registers, one partial row per CTA.
 // ---------------------------------------------------------------------------------------------
-template <int WPR>
+template <int WPR, bool SQ>
 __global__ void __launch_bounds__(WPR * 32) k_sort_sum_cta(const float* __restrict__ x, int ldx, int N, int count,
-                                                            float* __restrict__ partial) {
+                                                            float* __restrict__ partial, float* __restrict__ partial_sq) {
     __shared__ float xch[WPR * 1024];
     constexpr int E = 32, T_ = WPR * 32;
-    float acc[E];
+    float acc[E], acc_sq[SQ ? E : 1];
 #pragma unroll
     for (int r = 0; r < E; ++r) acc[r] = 0.0f;
+#pragma unroll
+    for (int r = 0; r < (SQ ? E : 1); ++r) acc_sq[r] = 0.0f;
     for (int row = blockIdx.x; row < count; row += gridDim.x) {
         const float* src = x + static_cast<size_t>(row) * ldx;
         float v[E];
@@ -350,11 +371,18 @@ __global__ void __launch_bounds__(WPR * 32) k_sort_sum_cta(const float* __restri
         cta_bitonic_sort<float, WPR>(v, xch);
 #pragma unroll
         for (int r = 0; r < E; ++r) acc[r] += v[r];
+        if (SQ) {
+#pragma unroll
+            for (int r = 0; r < E; ++r) acc_sq[SQ ? r : 0] = fmaf(v[r], v[r], acc_sq[SQ ? r : 0]);
+        }
     }
 #pragma unroll
     for (int r = 0; r < E; ++r) {
         const int idx = threadIdx.x * E + r;
-        if (idx < N) partial[static_cast<size_t>(blockIdx.x) * N + idx] = acc[r];
+        if (idx < N) {
+            partial[static_cast<size_t>(blockIdx.x) * N + idx] = acc[r];
+            if (SQ) partial_sq[static_cast<size_t>(blockIdx.x) * N + idx] = acc_sq[SQ ? r : 0];
+        }
     }
 }
 
@@ -417,10 +445,36 @@ constexpr int kColsumThreads = 256;
 
 __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* __restrict__ partial, int n_part, int N,
                                                                    double* sums, double inv_samples, DevState* st,
-                                                                   float* __restrict__ e_out, float* __restrict__ omega_out) {
+                                                                   float* __restrict__ e_out, float* __restrict__ omega_out,
+                                                                   const float* __restrict__ partial_sq,
+                                                                   float* __restrict__ std_out) {
     __shared__ double red[8][32];
     __shared__ bool is_last;
     const int col = blockIdx.x * 32 + (threadIdx.x & 31), slice = threadIdx.x >> 5;
+    if (partial_sq) {
+        // spread of each order statistic over the samples: sqrt(E[x^2] - E[x]^2), in seconds
+        double s1 = 0.0, s2 = 0.0;
+        if (col < N)
+            for (int p = slice; p < n_part; p += 8) {
+                s1 += static_cast<double>(partial[static_cast<size_t>(p) * N + col]);
+                s2 += static_cast<double>(partial_sq[static_cast<size_t>(p) * N + col]);
+            }
+        red[slice][threadIdx.x & 31] = s1;
+        __syncthreads();
+        double t1 = 0.0;
+        if (slice == 0)
+            for (int k = 0; k < 8; ++k) t1 += red[k][threadIdx.x];
+        __syncthreads();
+        red[slice][threadIdx.x & 31] = s2;
+        __syncthreads();
+        if (slice == 0 && col < N) {
+            double t2 = 0.0;
+            for (int k = 0; k < 8; ++k) t2 += red[k][threadIdx.x];
+            const double mean = t1 * inv_samples, var = t2 * inv_samples - mean * mean;
+            std_out[col] = static_cast<float>(static_cast<double>(st->scale) * sqrt(var > 0.0 ? var : 0.0));
+        }
+        __syncthreads();
+    }
     double s = 0.0;
     if (col < N) {
         int p = slice;

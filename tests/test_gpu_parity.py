@@ -402,6 +402,34 @@ def test_censored_push_imputes_from_the_truncated_predictive(name, S):
     assert e.value.code == binding.ERR_STATE
 
 
+@pytest.mark.parametrize("name,S", [("tiny", 1024), ("n158", 1024), ("n1024", 2048), ("n2175", 300)])
+def test_order_statistic_spread(name, S):
+    # the +-2 sigma bands of the paper's Fig. 3: standard deviation of each order statistic over the samples
+    wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 5)
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.predict()
+        gpu.get_order_stat_std()                            # not asked for
+    assert e.value.code == binding.ERR_STATE
+    plain = gpu.get_stats()[0]
+    orc.predict()
+    gpu.restore_state(_state_before(gpu, wl, name))         # same decision again, now with the squares
+    gpu.set_option("order_stat_std", 1)
+    code, c = gpu.predict()
+    sd = gpu.get_order_stat_std()
+    assert np.array_equal(gpu.get_stats()[0], plain)        # the means do not change
+    want = orc.last_std_sec
+    assert np.max(np.abs(sd - want)) <= 2e-3 * want.max()
+    assert np.all(sd >= 0)
+
+
+def _state_before(gpu, wl, name):
+    """Observation state of a fresh context that saw the same pushes and has made no decision."""
+    fresh = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 64, precision=0)
+    for x in inputs.workload_trace(wl, wl.window + 5):
+        fresh.push(x)
+    return fresh.save_state()
+
+
 def test_degenerate_and_equal_times():
     # every expected time negative -> c = N with the informational code; equal deterministic times -> c = N
     wl = inputs.WORKLOADS["tiny"]

@@ -544,3 +544,19 @@ def test_oracle_push_with_censoring_uses_the_last_decision():
     assert np.array_equal(pushed[~censored], observed[~censored])
     assert np.all(pushed[censored] >= observed[~censored].max())
     assert orc.predict()[0] == O.OK
+
+
+def test_order_statistic_spread_matches_closed_forms():
+    # two iid N(mu, sigma^2) times: Var(max) = Var(min) = sigma^2 (1 - 1/pi); one time: sigma itself
+    mu, sigma, S = 0.8, 0.25, 1 << 18
+    x = _predictive_samples(_constant_emission_weights(2, mu=mu, sigma=sigma), S)
+    sd = O.order_statistic_std(x)
+    want = sigma * math.sqrt(1.0 - 1.0 / math.pi)
+    assert np.all(np.abs(sd / want - 1.0) < 5.0 / math.sqrt(2 * S) * 1.5)
+    x1 = _predictive_samples(_constant_emission_weights(1, mu=mu, sigma=sigma), S)
+    assert abs(O.order_statistic_std(x1)[0] / sigma - 1.0) < 5.0 / math.sqrt(2 * S)
+    # the spread is about the position's own mean: shifting all times changes nothing
+    assert np.allclose(O.order_statistic_std(x + 3.0), sd, rtol=1e-9)
+    orc = _driven_oracle("tiny", 256)
+    orc.predict()
+    assert np.allclose(orc.last_std_sec, np.sort(orc.last_draws_sec, axis=1).std(axis=0), rtol=1e-12)
