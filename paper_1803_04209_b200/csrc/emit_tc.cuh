@@ -108,6 +108,63 @@ struct EmitArgs {
     int count, N, H, ldx;
 };
 
+// Epilogue of one 128 x 128 output tile for one warp: read its 32 lanes x 32 (+32) accumulator columns, hand the
+// accumulator back, add the biases, draw the noise and store x = mean + exp(logvar / 2) * eps.
+__device__ __forceinline__ void emit_epilogue_tile(const EmitArgs& a, uint32_t tmem_base, uint32_t acc, int q, int cg,
+                                                   int lane, int m0, int w0, uint32_t step, uint32_t bar_acc_empty) {
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + cg * 32;
+    const int row = m0 + q * 32 + lane;
+    const bool row_ok = row < a.count;
+    const uint32_t sample = a.sample_base + static_cast<uint32_t>(row);
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t mean_bits[16], logvar_bits[16];
+        tmem_ld16(taddr + 16 * half, mean_bits);
+        tmem_ld16(taddr + kBW + 16 * half, logvar_bits);
+        tmem_ld_wait();
+        if (half == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);    // accumulator is free again
+        }
+        const int jw = w0 + cg * 32 + 16 * half;
+        if (row_ok && jw < a.N) {
+            float* dst = a.x + static_cast<size_t>(row) * a.ldx + jw;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = jw + 4 * i;
+                if (j >= a.N) continue;
+                float eps[4];
+                normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
+                             a.key.seed_hi, eps);
+                float out[4];
+                if (j + 3 < a.N && (a.N & 3) == 0) {
+                    const float4 bm = __ldg(reinterpret_cast<const float4*>(a.b4 + j));
+                    const float4 bl = __ldg(reinterpret_cast<const float4*>(a.b4 + a.N + j));
+                    const float bmv[4] = {bm.x, bm.y, bm.z, bm.w}, blv[4] = {bl.x, bl.y, bl.z, bl.w};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        out[c] = fmaf(exp_half_fast(__uint_as_float(logvar_bits[4 * i + c]) + blv[c]), eps[c],
+                                      __uint_as_float(mean_bits[4 * i + c]) + bmv[c]);
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int jj = min(j + c, a.N - 1);
+                        const float mean = __uint_as_float(mean_bits[4 * i + c]) + __ldg(a.b4 + jj);
+                        const float logvar = __uint_as_float(logvar_bits[4 * i + c]) + __ldg(a.b4 + a.N + jj);
+                        out[c] = fmaf(exp_half_fast(logvar), eps[c], mean);
+                    }
+                }
+                if (j + 3 < a.N) {
+                    *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(out[0], out[1], out[2], out[3]);
+                } else {
+                    for (int c = 0; c < 4 && j + c < a.N; ++c) dst[4 * i + c] = out[c];
+                }
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__ CUtensorMap map_v,
                                                           const __grid_constant__ CUtensorMap map_w4, EmitArgs a) {
     extern __shared__ uint8_t smem_raw[];
@@ -231,47 +288,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__
             ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, a.st);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + cg * 32;
-            const int row = m0 + q * 32 + lane;
-            const bool row_ok = row < a.count;
-            const uint32_t sample = a.sample_base + static_cast<uint32_t>(row);
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t mean_bits[16], logvar_bits[16];
-                tmem_ld16(taddr + 16 * half, mean_bits);
-                tmem_ld16(taddr + kBW + 16 * half, logvar_bits);
-                tmem_ld_wait();
-                if (half == 1) {
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);    // accumulator is free again
-                }
-                const int jw = w0 + cg * 32 + 16 * half;
-                if (row_ok && jw < a.N) {
-                    float* dst = a.x + static_cast<size_t>(row) * a.ldx + jw;
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int j = jw + 4 * i;
-                        if (j >= a.N) continue;
-                        float eps[4];
-                        normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
-                                     a.key.seed_hi, eps);
-                        float out[4];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const int jj = min(j + c, a.N - 1);
-                            const float mean = __uint_as_float(mean_bits[4 * i + c]) + __ldg(a.b4 + jj);
-                            const float logvar = __uint_as_float(logvar_bits[4 * i + c]) + __ldg(a.b4 + a.N + jj);
-                            out[c] = fmaf(exp_half_fast(logvar), eps[c], mean);
-                        }
-                        if (j + 3 < a.N) {
-                            *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(out[0], out[1], out[2], out[3]);
-                        } else {
-                            for (int c = 0; c < 4 && j + c < a.N; ++c) dst[4 * i + c] = out[c];
-                        }
-                    }
-                }
-            }
+            emit_epilogue_tile(a, tmem_base, acc, q, cg, lane, m0, w0, step, bar_acc_empty);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }

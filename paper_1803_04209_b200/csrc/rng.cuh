@@ -25,12 +25,12 @@ __device__ __forceinline__ Philox4 philox4x32_10(uint32_t c0, uint32_t c1, uint3
     constexpr uint32_t kWeylA = 0x9E3779B9u, kWeylB = 0xBB67AE85u;
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
-        const uint32_t hi_a = __umulhi(kMulA, c0), lo_a = kMulA * c0;
-        const uint32_t hi_b = __umulhi(kMulB, c2), lo_b = kMulB * c2;
-        c0 = hi_b ^ c1 ^ k0;
-        c1 = lo_b;
-        c2 = hi_a ^ c3 ^ k1;
-        c3 = lo_a;
+        const unsigned long long prod_a = static_cast<unsigned long long>(kMulA) * c0;   // one wide multiply each
+        const unsigned long long prod_b = static_cast<unsigned long long>(kMulB) * c2;
+        c0 = static_cast<uint32_t>(prod_b >> 32) ^ c1 ^ k0;
+        c1 = static_cast<uint32_t>(prod_b);
+        c2 = static_cast<uint32_t>(prod_a >> 32) ^ c3 ^ k1;
+        c3 = static_cast<uint32_t>(prod_a);
         k0 += kWeylA;
         k1 += kWeylB;
     }
