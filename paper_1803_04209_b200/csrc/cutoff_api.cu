@@ -13,6 +13,7 @@
 #include "kernels_sort.cuh"
 #include "emit_tc.cuh"
 #include "chain_tc.cuh"
+#include "chain_tc32.cuh"
 
 using namespace cutoff;
 
@@ -69,6 +70,7 @@ struct cutoff_ctx {
     CUtensorMap map_w4{};           // TMA view of W4    [2N][H]
     bool use_tc = false;            // emission output layer on tensor cores
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
+    bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
     float* d_chain_image = nullptr; // swizzled tf32 operand tiles of the chain
 
     float* h_stage = nullptr;       // pinned [N]
@@ -238,8 +240,28 @@ void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
     c->launches += 1;
 }
 
+void launch_chain_tc32(cutoff_ctx* c, uint32_t sample_base, int count) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(tc::k_chain_tc32, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        attr_set = true;
+    }
+    tc::ChainTc32Args a;
+    const ModelDev& m = c->m;
+    a.image = c->d_chain_image;
+    a.bz = m.bz; a.b1 = m.b1; a.b3 = m.b3; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig; a.b2 = m.b2; a.z0 = m.z0;
+    a.hlr = c->d_hlr; a.st = c->d_state;
+    a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.round_v = 1; a.v_out = c->d_v;
+    const int tiles = ceil_div(count, 128);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    tc::k_chain_tc32<<<grid, tc::kChainTcThreads, tc::chain_tc32_smem_bytes(c->H, c->W), c->stream>>>(a);
+    c->launches += 1;
+}
+
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
     if (c->chain_tc) { launch_chain_tc(c, sample_base, count); return; }
+    if (c->chain_tc32) { launch_chain_tc32(c, sample_base, count); return; }
     const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
     switch (c->D) {
         case 4: launch_chain_t<4>(c, sample_base, count, smem); break;
@@ -470,6 +492,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
     c->chain_tc = c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
                   tc::chain_tc_smem_bytes(c->H, c->W) <= 227 * 1024;
+    c->chain_tc32 = c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
+                    (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W) <= 227 * 1024;
 
     size_t blob_floats = 0;
     for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
@@ -477,6 +501,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 3 * c->H * c->D));
     CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
+    if (c->chain_tc32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_mask, c->N));
@@ -608,6 +633,42 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
                 for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
                 for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + at(o, jj)] = tf32(w2[o * H + kb * 32 + jj]);
             }
+        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+
+    if (c->chain_tc32) {
+        // D = 32: six tiles of H x 32 tf32 values each -- Wz, W1, W3 as [H rows][32], Wmu and the two halves of W2 as
+        // H/32 K blocks of [32 rows][32] -- in the swizzled shared-memory layout, staged by the kernel phase by phase
+        auto tf32 = [](float f) {
+            uint32_t u;
+            std::memcpy(&u, &f, 4);
+            u = (u + 0x1000u) & 0xFFFFE000u;
+            std::memcpy(&f, &u, 4);
+            return f;
+        };
+        auto at = [](size_t row, size_t col) {
+            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
+        };
+        const size_t tile = H * 32;
+        std::vector<float> img(tc::chain_tc32_image_floats(c->H), 0.0f);
+        const float* wz = host.data() + off[8];
+        const float* w1 = host.data() + off[15];
+        const float* w3 = host.data() + off[19];
+        const float* wmu = host.data() + off[10];    // [32][H]
+        const float* w2 = host.data() + off[17];     // [64][H]: rows 0..31 mean, 32..63 log-variance
+        for (size_t n = 0; n < H; ++n)
+            for (size_t k = 0; k < 32; ++k) {
+                img[0 * tile + at(n, k)] = tf32(wz[n * 32 + k]);
+                img[1 * tile + at(n, k)] = tf32(w1[n * 32 + k]);
+                img[2 * tile + at(n, k)] = tf32(w3[n * 32 + k]);
+            }
+        for (size_t kb = 0; kb < H / 32; ++kb)
+            for (size_t jj = 0; jj < 32; ++jj)
+                for (size_t d = 0; d < 32; ++d) {
+                    img[3 * tile + kb * 1024 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
+                    img[4 * tile + kb * 1024 + at(d, jj)] = tf32(w2[d * H + kb * 32 + jj]);
+                    img[5 * tile + kb * 1024 + at(d, jj)] = tf32(w2[(32 + d) * H + kb * 32 + jj]);
+                }
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
 
