@@ -152,8 +152,9 @@ def run_reference(args, wl, weights, trace):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S": wl.S,
-                   "timed_samples_per_step": sample_S},
+        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S_per_gpu": wl.S,
+                   "parallelism": "samples x1", "timed_samples_per_step": sample_S,
+                   "timing": "host clock around the oracle's decision on the sampled rows"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
@@ -163,7 +164,7 @@ def run_reference(args, wl, weights, trace):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="n1024")

@@ -341,9 +341,10 @@ class CutoffOracle:
         rows = [self.samples(np.arange(k0, min(k0 + self.chunk, self.S)))   # rows are independent:
                 for k0 in range(0, self.S, self.chunk)]                     # chunking only bounds memory
         draws = np.concatenate(rows, axis=0)
+        ordered = np.sort(draws, axis=1, kind="stable")      # sorted once, used for the mean and for the spread
         self.last_draws_sec = s * draws
-        self.last_std_sec = s * order_statistic_std(draws)
-        expected = s * expected_order_statistics(draws)
+        self.last_std_sec = s * ordered.std(axis=0)
+        expected = s * ordered.mean(axis=0)
         omega = throughput(expected)
         c, degenerate = argmax_cutoff(omega)
         self.step += 1
