@@ -430,6 +430,23 @@ def _state_before(gpu, wl, name):
     return fresh.save_state()
 
 
+@pytest.mark.parametrize("N,D,H,lag,S,prec", [(1, 4, 32, 0, 300, 0), (3, 4, 32, 1, 257, 0), (5, 8, 64, 0, 129, 0),
+                                               (130, 16, 64, 0, 200, 1), (257, 16, 192, 2, 130, 1), (1025, 32, 96, 1, 140, 2)])
+def test_small_and_ragged_shapes(N, D, H, lag, S, prec):
+    # one worker, odd worker counts, a window of one vector, sample counts that leave ragged tiles
+    w = inputs.make_weights(N, D, H, seed=3, fan_in_ref=32, bf16=(prec == 2))
+    trace = inputs.make_trace(N, lag + 4, seed=9, sigma=0.2)
+    gpu = binding.Cutoff(N, D, H, lag, S, precision=prec, seed=SEED)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, lag, S, seed=SEED)
+    for x in trace:
+        gpu.push(x)
+        orc.push(x)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec])
+    c = assert_decision_close(gpu, orc.predict(), N)
+    assert 1 <= c <= N
+
+
 def test_degenerate_and_equal_times():
     # every expected time negative -> c = N with the informational code; equal deterministic times -> c = N
     wl = inputs.WORKLOADS["tiny"]
