@@ -32,7 +32,7 @@ struct TensorSpec { const char* name; size_t rows, cols; };
 struct cutoff_ctx {
     cutoff_config cfg{};
     int N = 0, D = 0, H = 0, W = 0, S = 0;
-    int ldx = 0;            // leading dimension of the sample matrix (N rounded up to 4)
+    int ldx = 0;            // leading dimension of the sample matrix (N rounded up to 8: rows start on 32 bytes)
     int P = 0;              // sort width: N rounded up to a power of two, at least 32
     int sm_count = 0;
     int chunk_rows = 0;     // samples per pass through chain -> emission -> sort
@@ -459,7 +459,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     if (!c) return CUTOFF_ERR_NOMEM;
     c->cfg = *cfg;
     c->N = cfg->n_workers; c->D = cfg->latent_dim; c->H = cfg->hidden; c->W = cfg->lag + 1; c->S = cfg->n_samples;
-    c->ldx = (c->N + 3) & ~3;
+    c->ldx = (c->N + 7) & ~7;
     c->P = next_pow2(c->N) < 32 ? 32 : next_pow2(c->N);
     c->stream = static_cast<cudaStream_t>(cfg->stream);
 

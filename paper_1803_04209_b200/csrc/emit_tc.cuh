@@ -37,7 +37,8 @@ constexpr int kEpiWarps = 16;
 constexpr int kThreads = (2 + kEpiWarps) * 32;
 constexpr int kTmemCols = 512;
 constexpr int kAccCols = 2 * kBW;                // 256 columns per accumulator
-constexpr size_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kBiasBytes = kEpiWarps * 64 * 4;   // per epilogue warp: 32 mean + 32 log-variance biases of its columns
+constexpr size_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/ + kBiasBytes;
 
 // instruction descriptor: D = f32, A = B = tf32, both K-major, N = 256, M = 128
 constexpr uint32_t kInstrDesc = (1u << 4) | (2u << 7) | (2u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
@@ -99,6 +100,12 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, uint32_t (&r)[8]) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// One 256-bit store: eight consecutive floats at a 32-byte aligned address.
+__device__ __forceinline__ void store8(float* p, const float* v) {
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
+
 struct EmitArgs {
     const float* b4;        // [2N]
     float* x;               // [count][ldx]
@@ -110,8 +117,10 @@ struct EmitArgs {
 
 // Epilogue of one 128 x 128 output tile for one warp: read its 32 lanes x 32 (+32) accumulator columns, hand the
 // accumulator back, add the biases, draw the noise and store x = mean + exp(logvar / 2) * eps.
+// bias_s: this warp's 32 mean biases, then its 32 log-variance biases, in shared memory (zero beyond worker N).
 __device__ __forceinline__ void emit_epilogue_tile(const EmitArgs& a, uint32_t tmem_base, uint32_t acc, int q, int cg,
-                                                   int lane, int m0, int w0, uint32_t step, uint32_t bar_acc_empty) {
+                                                   int lane, int m0, int w0, uint32_t step, uint32_t bar_acc_empty,
+                                                   const float* bias_s) {
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + cg * 32;
     const int row = m0 + q * 32 + lane;
     const bool row_ok = row < a.count;
@@ -130,6 +139,7 @@ __device__ __forceinline__ void emit_epilogue_tile(const EmitArgs& a, uint32_t t
         const int jw = w0 + cg * 32 + 16 * half;
         if (row_ok && jw < a.N) {
             float* dst = a.x + static_cast<size_t>(row) * a.ldx + jw;
+            float out[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int j = jw + 4 * i;
@@ -137,28 +147,31 @@ __device__ __forceinline__ void emit_epilogue_tile(const EmitArgs& a, uint32_t t
                 float eps[4];
                 normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
                              a.key.seed_hi, eps);
-                float out[4];
-                if (j + 3 < a.N && (a.N & 3) == 0) {
-                    const float4 bm = __ldg(reinterpret_cast<const float4*>(a.b4 + j));
-                    const float4 bl = __ldg(reinterpret_cast<const float4*>(a.b4 + a.N + j));
-                    const float bmv[4] = {bm.x, bm.y, bm.z, bm.w}, blv[4] = {bl.x, bl.y, bl.z, bl.w};
+                const float4 bm = *reinterpret_cast<const float4*>(bias_s + 16 * half + 4 * i);
+                const float4 bl = *reinterpret_cast<const float4*>(bias_s + 32 + 16 * half + 4 * i);
+                const float bmv[4] = {bm.x, bm.y, bm.z, bm.w}, blv[4] = {bl.x, bl.y, bl.z, bl.w};
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        out[c] = fmaf(exp_half_fast(__uint_as_float(logvar_bits[4 * i + c]) + blv[c]), eps[c],
-                                      __uint_as_float(mean_bits[4 * i + c]) + bmv[c]);
-                } else {
+                for (int c = 0; c < 4; ++c)
+                    out[4 * i + c] = fmaf(exp_half_fast(__uint_as_float(logvar_bits[4 * i + c]) + blv[c]), eps[c],
+                                          __uint_as_float(mean_bits[4 * i + c]) + bmv[c]);
+            }
+            // a thread owns 16 consecutive workers of its sample: two 32-byte stores (whole sectors; the row pitch
+            // is a multiple of 8 floats), 16-byte or scalar stores on the ragged edge
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int jj = min(j + c, a.N - 1);
-                        const float mean = __uint_as_float(mean_bits[4 * i + c]) + __ldg(a.b4 + jj);
-                        const float logvar = __uint_as_float(logvar_bits[4 * i + c]) + __ldg(a.b4 + a.N + jj);
-                        out[c] = fmaf(exp_half_fast(logvar), eps[c], mean);
-                    }
+            for (int p = 0; p < 2; ++p) {
+                if (jw + 8 * p + 7 < a.N) {
+                    store8(dst + 8 * p, out + 8 * p);
+                    continue;
                 }
-                if (j + 3 < a.N) {
-                    *reinterpret_cast<float4*>(dst + 4 * i) = make_float4(out[0], out[1], out[2], out[3]);
-                } else {
-                    for (int c = 0; c < 4 && j + c < a.N; ++c) dst[4 * i + c] = out[c];
+#pragma unroll
+                for (int i = 2 * p; i < 2 * p + 2; ++i) {
+                    const int ji = jw + 4 * i;
+                    if (ji + 3 < a.N) {
+                        *reinterpret_cast<float4*>(dst + 4 * i) =
+                            make_float4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+                    } else {
+                        for (int c = 0; c < 4 && ji + c < a.N; ++c) dst[4 * i + c] = out[4 * i + c];
+                    }
                 }
             }
         }
@@ -178,6 +191,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__
     uint8_t* gen = smem_raw + (tiles - raw) + kStages * kStageBytes;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + 8 * (2 * kStages + 5));
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 8 * (2 * kStages + 5) + 8);
+    float* bias_all = reinterpret_cast<float*>(gen + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tiles_w = ceil_div(a.N, kBW);
@@ -281,14 +295,26 @@ __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__
         // ---------------- epilogue ---------------------------------------------------------------
         const int q = warp & 3, cg = (warp - 2) >> 2;
         const uint32_t step = a.st->step;
+        float* bias_s = bias_all + (warp - 2) * 64;
+        int w_staged = -1;
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
         for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
             const int m0 = (t / n_tiles_w) * kBM, w0 = (t % n_tiles_w) * kBW;
+            if (w0 != w_staged) {                       // biases of this warp's 32 workers, read once per worker tile
+                const int j = w0 + cg * 32 + lane;
+                const float bm = j < a.N ? __ldg(a.b4 + j) : 0.f;
+                const float bl = j < a.N ? __ldg(a.b4 + a.N + j) : 0.f;
+                __syncwarp();                           // the previous tile's readers are done
+                bias_s[lane] = bm;
+                bias_s[32 + lane] = bl;
+                __syncwarp();
+                w_staged = w0;
+            }
             ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, a.st);
             if (!ok) break;
             tc_fence_after();
-            emit_epilogue_tile(a, tmem_base, acc, q, cg, lane, m0, w0, step, bar_acc_empty);
+            emit_epilogue_tile(a, tmem_base, acc, q, cg, lane, m0, w0, step, bar_acc_empty, bias_s);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
