@@ -41,9 +41,13 @@ networks (ReLU / tanh with dense random weights) have no closed form:
 **parity unpinned** for ``encoder`` and ``guide_chain`` beyond those special
 cases.
 
-Model variant: transition and emission are one-hidden-layer ReLU MLPs with a
-(mean, log-variance) head.  The paper's gated transition and softplus scale
-networks are not built here.
+Model variants.  "compact": transition and emission are one-hidden-layer ReLU
+MLPs with a (mean, log-variance) head (``transition`` / ``emission``).
+"literal": the networks as Section 3.1.3 prints them -- the gated transition
+G, H and the emission I = MLP_2(z, Identity, Identity), J = MLP_2(I, ReLU,
+Softplus) (``transition_gated`` / ``emission_literal``); there the second
+argument of N(.,.) is taken as a standard deviation, like the guide's sigma.
+A weight dictionary that holds "Wg1" selects the literal variant.
 """
 from __future__ import annotations
 
@@ -210,17 +214,59 @@ def emission(z: np.ndarray, w: dict, eps: np.ndarray) -> np.ndarray:
     return mean + np.exp(0.5 * logvar) * eps
 
 
+def sigmoid(v):
+    return 1.0 / (1.0 + np.exp(-v))
+
+
+def transition_gated(z: np.ndarray, w: dict, eps: np.ndarray) -> np.ndarray:
+    """The gated transition of Section 3.1.3, z_{T+1} = G + H * eps with
+
+        g = MLP_2(z, ReLU, Sigmoid)          h = MLP_2(z, ReLU, Identity)
+        G = (1 - g) * MLP_1(z, Identity) + g * h
+        H = MLP_1(ReLU(G), Softplus)         (a standard deviation)
+    """
+    w = _f64(w)
+    g = sigmoid(relu(z @ w["Wg1"].T + w["bg1"]) @ w["Wg2"].T + w["bg2"])
+    h = relu(z @ w["Wh1"].T + w["bh1"]) @ w["Wh2"].T + w["bh2"]
+    G = (1.0 - g) * (z @ w["Wl"].T + w["bl"]) + g * h
+    H = softplus(relu(G) @ w["Ws"].T + w["bs"])
+    return G + H * eps
+
+
+def emission_literal(z: np.ndarray, w: dict, eps: np.ndarray) -> np.ndarray:
+    """The emission of Section 3.1.3, x_{T+1} = I + J * eps with
+
+        I = MLP_2(z, Identity, Identity)     (two affine layers: the mean of every worker)
+        J = MLP_2(I, ReLU, Softplus)         (a standard deviation, computed from the mean)
+    """
+    w = _f64(w)
+    I = (z @ w["Wi1"].T + w["bi1"]) @ w["Wi2"].T + w["bi2"]
+    J = softplus(relu(I @ w["Wj1"].T + w["bj1"]) @ w["Wj2"].T + w["bj2"])
+    return I + J * eps
+
+
+def is_literal(w: dict) -> bool:
+    return "Wg1" in w
+
+
+def n_workers(w: dict) -> int:
+    return w["bi2"].shape[0] if is_literal(w) else w["b4"].shape[0] // 2
+
+
 def sample_runtimes(w: dict, xhat: np.ndarray, seed: int, step: int, k) -> np.ndarray:
     """Posterior-predictive draws x^(k)_{T+1} (normalised units), one row per sample index."""
     k = np.asarray(k, dtype=np.int64).reshape(-1)
     W = xhat.shape[0]
     D = w["z0"].shape[0]
-    N = w["b4"].shape[0] // 2
+    N = n_workers(w)
     a, b = encoder(xhat, w)
     eps_q = np.stack([normals(seed, step, t, k, D) for t in range(W)], axis=1)
     z_T = guide_chain(a, b, w, eps_q)
-    z_next = transition(z_T, w, normals(seed, step, STREAM_TRANSITION, k, D))
-    return emission(z_next, w, normals(seed, step, STREAM_EMISSION, k, N))
+    eps_tr = normals(seed, step, STREAM_TRANSITION, k, D)
+    eps_em = normals(seed, step, STREAM_EMISSION, k, N)
+    if is_literal(w):
+        return emission_literal(transition_gated(z_T, w, eps_tr), w, eps_em)
+    return emission(transition(z_T, w, eps_tr), w, eps_em)
 
 
 # ----------------------------------------------------------------------------
@@ -303,7 +349,7 @@ class CutoffOracle:
         self.S = n_samples
         self.seed = seed
         self.chunk = chunk
-        self.N = weights["b4"].shape[0] // 2
+        self.N = n_workers(weights)
         self.reset()
 
     def reset(self):

@@ -262,14 +262,11 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc32(ChainTc32Args
                         if (lane == 0) mbar_arrive(bar_h + 8 * b);
                         ++nu;
                     } else if (k < a.count) {
-                        float4* out = reinterpret_cast<float4*>(a.v_out + static_cast<size_t>(k) * H + col0);
-                        float4 o0 = make_float4(h[0], h[1], h[2], h[3]), o1 = make_float4(h[4], h[5], h[6], h[7]);
                         if (a.round_v) {
-                            o0.x = tf32_rna(o0.x); o0.y = tf32_rna(o0.y); o0.z = tf32_rna(o0.z); o0.w = tf32_rna(o0.w);
-                            o1.x = tf32_rna(o1.x); o1.y = tf32_rna(o1.y); o1.z = tf32_rna(o1.z); o1.w = tf32_rna(o1.w);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) h[i] = tf32_rna(h[i]);
                         }
-                        out[0] = o0;
-                        out[1] = o1;
+                        store8(a.v_out + static_cast<size_t>(k) * H + col0, h);          // one whole 32-byte sector
                     }
                 }
                 if (!ok || ph > W) continue;

@@ -43,6 +43,30 @@ def tensor_shapes(N: int, D: int, H: int) -> dict:
     }
 
 
+# The networks as Section 3.1.3 prints them ("literal" variant): the guide tensors
+# are the same; the generative model has
+#   gated transition:  gate Wg1 bg1 Wg2 bg2 | proposal Wh1 bh1 Wh2 bh2 | linear Wl bl | scale Ws bs
+#   emission:          mean Wi1 bi1 Wi2 bi2 (two affine layers) | scale Wj1 bj1 Wj2 bj2 (input: the mean)
+GUIDE_TENSORS = TENSOR_ORDER[:15]
+TENSOR_ORDER_LITERAL = GUIDE_TENSORS + (
+    "Wg1", "bg1", "Wg2", "bg2", "Wh1", "bh1", "Wh2", "bh2", "Wl", "bl", "Ws", "bs",
+    "Wi1", "bi1", "Wi2", "bi2", "Wj1", "bj1", "Wj2", "bj2",
+)
+
+
+def tensor_shapes_literal(N: int, D: int, H: int) -> dict:
+    base = tensor_shapes(N, D, H)
+    shapes = {k: base[k] for k in GUIDE_TENSORS}
+    shapes.update({
+        "Wg1": (H, D), "bg1": (H,), "Wg2": (D, H), "bg2": (D,),
+        "Wh1": (H, D), "bh1": (H,), "Wh2": (D, H), "bh2": (D,),
+        "Wl": (D, D), "bl": (D,), "Ws": (D, D), "bs": (D,),
+        "Wi1": (H, D), "bi1": (H,), "Wi2": (N, H), "bi2": (N,),
+        "Wj1": (H, N), "bj1": (H,), "Wj2": (N, H), "bj2": (N,),
+    })
+    return shapes
+
+
 def round_to_bf16(a: np.ndarray) -> np.ndarray:
     """Round fp32 values to the nearest bf16-representable fp32 (ties to even)."""
     u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32).astype(np.uint64)
@@ -92,6 +116,33 @@ def make_weights(N: int, D: int, H: int, seed: int = 0, std: float = 0.1,
     return w
 
 
+def make_weights_literal(N: int, D: int, H: int, seed: int = 0, std: float = 0.1,
+                         fan_in_ref: int | None = None, offsets: bool = True) -> dict:
+    """Random-initialised weights of the literal variant, drawn like `make_weights`.
+
+    ``offsets=True`` moves the untrained model into the regime of a fitted one:
+      emission mean        last layer and bias halved, then bias += 0.5
+      emission scale       bias += softplus^-1(0.05)   (noise of about 0.05)
+      transition scale     bias += softplus^-1(0.1)    (a slowly moving latent)
+    """
+    rng = np.random.Generator(np.random.Philox(seed))
+    w = {}
+    for name, shape in tensor_shapes_literal(N, D, H).items():
+        if name in ("a0", "b0", "z0"):
+            w[name] = np.zeros(shape, dtype=np.float32)
+            continue
+        sd = std
+        if fan_in_ref is not None and len(shape) == 2 and shape[1] > fan_in_ref:
+            sd = std * math.sqrt(fan_in_ref / shape[1])
+        w[name] = (rng.standard_normal(shape) * sd).astype(np.float32)
+    if offsets:
+        w["Wi2"] *= np.float32(0.5)
+        w["bi2"] = w["bi2"] * np.float32(0.5) + np.float32(0.5)
+        w["bj2"] += np.float32(math.log(math.expm1(0.05)))
+        w["bs"] += np.float32(math.log(math.expm1(0.1)))
+    return w
+
+
 @dataclass(frozen=True)
 class Workload:
     name: str
@@ -133,6 +184,10 @@ WORKLOADS = {
                       trace_seed=6, trace=dict(sigma=0.3, groups=32, stay=0.9, slowdown=2.0,
                                                straggler_p=0.01, straggler="exp", straggler_scale=1.5)),
 }
+
+
+def workload_weights_literal(wl: Workload, offsets: bool = True) -> dict:
+    return make_weights_literal(wl.N, wl.D, wl.H, seed=wl.weight_seed, std=0.1, fan_in_ref=32, offsets=offsets)
 
 
 def workload_weights(wl: Workload, offsets: bool = True) -> dict:
