@@ -48,7 +48,7 @@ def compare_exchanges(n_pow2: int) -> int:
     return (n_pow2 // 2) * lg * (lg + 1) // 2
 
 
-def stage_work(wl, S):
+def stage_work(wl, S, literal=False):
     """Algorithmic work of one decision per stage: (kind, amount).  'alu' counts one lane-operation per
     fused multiply-add or per min / max; 'tensor' counts floating-point operations (2 per multiply-add)."""
     N, D, H, W = wl.N, wl.D, wl.H, wl.window
@@ -57,6 +57,9 @@ def stage_work(wl, S):
         p *= 2
     chain = S * (W * (2 * D * H + D * D) + 3 * D * H + D * H)
     emit_macs = S * H * 2 * N
+    if literal:      # gate and proposal (2 x 2DH), linear map and scale (2 x D^2), first emission layer; three N x H products
+        chain = S * (W * (2 * D * H + D * D) + 4 * D * H + 2 * D * D + D * H)
+        emit_macs = S * H * 3 * N
     return {
         "encoder": ("alu", 2 * W * (N * H + H * H)),
         "chain": ("alu", chain),
@@ -152,8 +155,8 @@ def run_reference(args, wl, weights, trace):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S_per_gpu": wl.S,
-                   "parallelism": "samples x1", "timed_samples_per_step": sample_S,
+        "config": {"workload": wl.name, "variant": args.variant, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag,
+                   "S_per_gpu": wl.S, "parallelism": "samples x1", "timed_samples_per_step": sample_S,
                    "timing": "host clock around the oracle's decision on the sampled rows"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -168,6 +171,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="n1024")
+    ap.add_argument("--variant", default="compact", choices=["compact", "literal"],
+                    help="compact: one-hidden-layer MLPs with (mean, log-variance) heads; literal: the gated "
+                         "transition and the emission networks I, J as the paper prints them")
     ap.add_argument("--samples", type=int, default=0, help="override S (for profiling small cases)")
     ap.add_argument("--pass-rows", type=int, default=0)
     ap.add_argument("--reference-samples", type=int, default=4096)
@@ -184,7 +190,8 @@ def main():
     if args.samples:
         import dataclasses
         wl = dataclasses.replace(wl, S=args.samples)
-    weights = inputs.workload_weights(wl)
+    literal = args.variant == "literal"
+    weights = inputs.workload_weights_literal(wl) if literal else inputs.workload_weights(wl)
     trace = inputs.workload_trace(wl, min(wl.history, 64) + args.steps + args.warmup + 8)
 
     if args.impl == "reference":
@@ -209,7 +216,7 @@ def main():
     shard = sharding.shard_config(rank, world, wl.S)
     ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, shard["n_samples"], precision=wl.precision, seed=2024,
                          device=local_rank, stream=stream.cuda_stream, sample_offset=shard["sample_offset"],
-                         total_samples=shard["total_samples"])
+                         total_samples=shard["total_samples"], flags=binding.FLAG_LITERAL if literal else 0)
     shared = sharding.ShardedDecision(ctx, device="cuda") if world > 1 else None
     ctx.load_weights(weights)
     if args.pass_rows:
@@ -317,7 +324,7 @@ def main():
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except OSError:
         pass
-    work = stage_work(wl, wl.S)
+    work = stage_work(wl, wl.S, literal)
     stage_avg = {k: v / args.steps for k, v in stage_ms.items()}
     dominant = max(stage_avg, key=stage_avg.get)
     kind, amount = work[dominant]
@@ -337,7 +344,7 @@ def main():
         peak_src = "148 SMs x 128 fp32 lanes x max SM clock"
         bound = "alu"
     achieved = amount / dur / 1e12
-    traffic = NCU_TRAFFIC.get((wl.name, dominant))
+    traffic = None if literal else NCU_TRAFFIC.get((wl.name, dominant))
     roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
                 "frac": achieved / peak, "traffic": traffic["bytes_per_sample"] * wl.S if traffic else None,
                 "traffic_source": traffic["source"] if traffic else None,
@@ -355,8 +362,8 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": PRECISION_NAMES[wl.precision], "data": "synthetic",
-        "config": {"workload": wl.name, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag, "S_per_gpu": wl.S,
-                   "parallelism": f"samples x{world}", "l2": "flushed between timed steps (256 MiB write)",
+        "config": {"workload": wl.name, "variant": args.variant, "N": wl.N, "D": wl.D, "H": wl.H, "lag": wl.lag,
+                   "S_per_gpu": wl.S, "parallelism": f"samples x{world}", "l2": "flushed between timed steps (256 MiB write)",
                    "timing": "CUDA events per step on the library's stream"},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
                 "h2d_bytes_per_step": 4 * wl.N, "d2h_bytes_per_step": 40 + 8 * wl.N},

@@ -22,8 +22,10 @@
  *      averaged over the samples (Section 3.1.1, last paragraph);
  *   5. Omega(c) = c / E[x~_(c)] and c* = argmax_c Omega(c) (Section 3).
  *
- * Model variant: transition and emission are one-hidden-layer ReLU MLPs whose
- * heads give a mean and a log-variance.  All noise comes from Philox4x32-10
+ * Model variants: by default transition and emission are one-hidden-layer ReLU
+ * MLPs whose heads give a mean and a log-variance; with CUTOFF_FLAG_LITERAL they
+ * are the gated transition and the emission networks I, J as Section 3.1.3 prints
+ * them.  All noise comes from Philox4x32-10
  * (Salmon et al., SC'11) and the basic Box-Muller transform, addressed by
  * (seed, decision number, stage, sample, element), so results do not depend on
  * how the work is split over threads or GPUs.
@@ -71,7 +73,9 @@ enum {
 };
 
 enum {
-    CUTOFF_FLAG_GRAPH = 1       /* replay push+predict as one captured CUDA graph                  */
+    CUTOFF_FLAG_GRAPH = 1,      /* replay push+predict as one captured CUDA graph                  */
+    CUTOFF_FLAG_LITERAL = 2     /* the generative model exactly as Section 3.1.3 prints it (gated
+                                   transition, emission I / J); see cutoff_load_weights            */
 };
 
 typedef struct {
@@ -106,6 +110,16 @@ void cutoff_destroy(cutoff_ctx* ctx);
  *   Wz[HxD] bz[H] Wmu[DxH] bmu[D] Wsig[DxD] bsig[D] z0[D]             (combiner, mu_q, sigma_q)
  *   W1[HxD] b1[H] W2[2DxH] b2[2D]                                     (transition; rows D.. = log-variance)
  *   W3[HxD] b3[H] W4[2NxH] b4[2N]                                     (emission;   rows N.. = log-variance)
+ * A context created with CUTOFF_FLAG_LITERAL takes the networks as Section 3.1.3 prints them instead:
+ * the header's last word is 1, the guide tensors (first two lines above) are the same, and then follow
+ *   Wg1[HxD] bg1[H] Wg2[DxH] bg2[D]     gate      g = MLP_2(z, ReLU, Sigmoid)
+ *   Wh1[HxD] bh1[H] Wh2[DxH] bh2[D]     proposal  h = MLP_2(z, ReLU, Identity)
+ *   Wl[DxD] bl[D]                       G = (1 - g) * (Wl z + bl) + g * h
+ *   Ws[DxD] bs[D]                       H = Softplus(Ws ReLU(G) + bs)            z' = G + H * eps
+ *   Wi1[HxD] bi1[H] Wi2[NxH] bi2[N]     I = Wi2 (Wi1 z' + bi1) + bi2             (two affine layers)
+ *   Wj1[HxN] bj1[H] Wj2[NxH] bj2[N]     J = Softplus(Wj2 ReLU(Wj1 I + bj1) + bj2)   x = I + J * eps
+ * where H and J are standard deviations.  With a tensor-core precision the three products over N
+ * (Wi2, Wj1, Wj2) run on the tensor cores with tf32 operands (weights first rounded to bf16 for BF16W).
  * The blob is copied; the caller keeps ownership.  Errors: BAD_ARG, BAD_BLOB (size, magic or
  * dimensions do not match the context, or a value is not finite), CUDA. */
 int cutoff_load_weights(cutoff_ctx* ctx, const void* blob, size_t nbytes);

@@ -11,7 +11,7 @@ import struct
 
 import numpy as np
 
-from .inputs import TENSOR_ORDER, tensor_shapes
+from .inputs import TENSOR_ORDER, TENSOR_ORDER_LITERAL, tensor_shapes, tensor_shapes_literal
 
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(PKG_DIR, "libcutoff.so")
@@ -22,6 +22,7 @@ ERR_UNSUPPORTED, ERR_NOMEM, ERR_STATE, ERR_TIMEOUT, ERR_TOO_LARGE = -5, -6, -7, 
 STATIC_MAX_N = 1024
 PRECISION_FP32, PRECISION_TF32, PRECISION_BF16W = 0, 1, 2
 FLAG_GRAPH = 1
+FLAG_LITERAL = 2
 BLOB_MAGIC = 0x31465443
 
 EXPORTS = (
@@ -108,10 +109,15 @@ def strerror(code: int) -> str:
 
 
 def pack_weights(weights: dict, N: int, D: int, H: int) -> bytes:
-    """Serialise a weight dictionary into the blob cutoff_load_weights expects."""
-    shapes = tensor_shapes(N, D, H)
-    parts = [struct.pack("<6I", BLOB_MAGIC, 1, N, D, H, 0)]
-    for name in TENSOR_ORDER:
+    """Serialise a weight dictionary into the blob cutoff_load_weights expects.
+
+    A dictionary that holds "Wg1" is the literal variant (gated transition, emission I / J): its blob
+    carries 1 in the header's last word and goes to a context created with FLAG_LITERAL.
+    """
+    literal = "Wg1" in weights
+    shapes = tensor_shapes_literal(N, D, H) if literal else tensor_shapes(N, D, H)
+    parts = [struct.pack("<6I", BLOB_MAGIC, 1, N, D, H, 1 if literal else 0)]
+    for name in (TENSOR_ORDER_LITERAL if literal else TENSOR_ORDER):
         a = np.ascontiguousarray(weights[name], dtype=np.float32)
         if a.shape != shapes[name]:
             raise ValueError(f"{name}: shape {a.shape}, expected {shapes[name]}")

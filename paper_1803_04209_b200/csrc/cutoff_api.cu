@@ -14,6 +14,8 @@
 #include "emit_tc.cuh"
 #include "chain_tc.cuh"
 #include "chain_tc32.cuh"
+#include "kernels_literal.cuh"
+#include "gemm_tc.cuh"
 
 using namespace cutoff;
 
@@ -68,6 +70,14 @@ struct cutoff_ctx {
 
     CUtensorMap map_v{};            // TMA view of d_v   [alloc_rows][H]
     CUtensorMap map_w4{};           // TMA view of W4    [2N][H]
+
+    bool literal = false;           // the networks as Section 3.1.3 prints them (CUTOFF_FLAG_LITERAL)
+    LiteralDev lit{};
+    float* d_I = nullptr;           // [alloc_rows][ldx]  emission mean I (padding columns stay zero)
+    float* d_r = nullptr;           // [alloc_rows][H]    hidden layer of the emission scale
+    float* d_Wj1p = nullptr;        // [H][ldx]           Wj1 with rows padded with zeros to ldx
+    CUtensorMap map_I{}, map_r{};   // TMA views of d_I [alloc_rows][N] and d_r [alloc_rows][H]
+    CUtensorMap map_wi2{}, map_wj1{}, map_wj2{};
     bool use_tc = false;            // emission output layer on tensor cores
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
     bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
@@ -117,6 +127,22 @@ std::vector<TensorSpec> tensor_specs(size_t N, size_t D, size_t H) {
     };
 }
 
+// The literal variant: the guide tensors (the first 15) are the same, then the gated transition and the
+// emission networks I and J.
+std::vector<TensorSpec> tensor_specs_literal(size_t N, size_t D, size_t H) {
+    std::vector<TensorSpec> v = tensor_specs(N, D, H);
+    v.resize(15);
+    const TensorSpec rest[] = {
+        {"Wg1", H, D}, {"bg1", 1, H}, {"Wg2", D, H}, {"bg2", 1, D},
+        {"Wh1", H, D}, {"bh1", 1, H}, {"Wh2", D, H}, {"bh2", 1, D},
+        {"Wl", D, D}, {"bl", 1, D}, {"Ws", D, D}, {"bs", 1, D},
+        {"Wi1", H, D}, {"bi1", 1, H}, {"Wi2", N, H}, {"bi2", 1, N},
+        {"Wj1", H, N}, {"bj1", 1, H}, {"Wj2", N, H}, {"bj2", 1, N},
+    };
+    v.insert(v.end(), std::begin(rest), std::end(rest));
+    return v;
+}
+
 int next_pow2(int n) {
     int p = 1;
     while (p < n) p <<= 1;
@@ -124,6 +150,7 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
+    cudaFree(c->d_I); cudaFree(c->d_r); cudaFree(c->d_Wj1p);
     cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_WhR); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
     if (c->h_mask) cudaFreeHost(c->h_mask); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
@@ -259,7 +286,30 @@ void launch_chain_tc32(cutoff_ctx* c, uint32_t sample_base, int count) {
     c->launches += 1;
 }
 
+template <int D>
+void launch_chain_literal_t(cutoff_ctx* c, uint32_t sample_base, int count) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(k_chain_literal<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+        attr_set = true;
+    }
+    const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
+    k_chain_literal<D><<<ceil_div(count, ChainShape<D>::kSamplesPerCta), ChainShape<D>::kThreads, smem, c->stream>>>(
+        c->m, c->lit, c->d_hlr, c->d_state, key, sample_base, count, c->use_tc ? 1 : 0, c->d_v);
+}
+
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
+    if (c->literal) {
+        switch (c->D) {
+            case 4: launch_chain_literal_t<4>(c, sample_base, count); break;
+            case 8: launch_chain_literal_t<8>(c, sample_base, count); break;
+            case 16: launch_chain_literal_t<16>(c, sample_base, count); break;
+            default: launch_chain_literal_t<32>(c, sample_base, count); break;
+        }
+        c->launches += 1;
+        return;
+    }
     if (c->chain_tc) { launch_chain_tc(c, sample_base, count); return; }
     if (c->chain_tc32) { launch_chain_tc32(c, sample_base, count); return; }
     const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
@@ -274,7 +324,7 @@ void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
 
 // 2-D fp32 tensor map over a row-major [rows][cols] matrix, boxes of 128 rows x 32 columns
 // (one 128-byte-swizzled K-major operand tile).  The driver entry point is looked up at run time.
-int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t rows, uint64_t cols) {
+int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t rows, uint64_t cols, uint64_t ld = 0) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -290,7 +340,7 @@ int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t r
         encode = reinterpret_cast<EncodeFn>(fn);
     }
     const cuuint64_t dims[2] = {cols, rows};
-    const cuuint64_t strides[1] = {cols * sizeof(float)};
+    const cuuint64_t strides[1] = {(ld ? ld : cols) * sizeof(float)};
     const cuuint32_t box[2] = {tc::kBK, tc::kBM};
     const cuuint32_t elem[2] = {1, 1};
     const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box,
@@ -319,7 +369,50 @@ void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
     c->launches += 1;
 }
 
+// Literal emission (Section 3.1.3): I = u Wi2^T + bi2, r = relu(I Wj1^T + bj1), x = I + softplus(r Wj2^T + bj2) * eps.
+template <int EPI>
+void launch_gemm_tc(cutoff_ctx* c, const CUtensorMap& map_a, const CUtensorMap& map_b, const tc::GemmTcArgs& a) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(tc::k_gemm_tc<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
+        attr_set = true;
+    }
+    const int tiles = ceil_div(a.Nout, tc::kGemmBN) * ceil_div(a.M, tc::kBM);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    tc::k_gemm_tc<EPI><<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(map_a, map_b, a);
+    c->launches += 1;
+}
+
+void launch_emission_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
+    const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    const LiteralDev& l = c->lit;
+    if (c->use_tc) {
+        tc::GemmTcArgs a{};
+        a.st = c->d_state; a.key = key; a.sample_base = sample_base; a.M = count;
+        a.bias = l.bi2; a.out = c->d_I; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H;
+        launch_gemm_tc<kEpiAffine>(c, c->map_v, c->map_wi2, a);
+        a.bias = l.bj1; a.out = c->d_r; a.ld_out = c->H; a.Nout = c->H; a.K = c->N; a.round_out = 1;
+        launch_gemm_tc<kEpiRelu>(c, c->map_I, c->map_wj1, a);
+        a.bias = l.bj2; a.add = c->d_I; a.out = c->d_x; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H; a.round_out = 0;
+        launch_gemm_tc<kEpiScaleNoise>(c, c->map_r, c->map_wj2, a);
+        return;
+    }
+    GemmFmaArgs a{};
+    a.st = c->d_state; a.key = key; a.sample_base = sample_base; a.M = count;
+    a.A = c->d_v; a.lda = c->H; a.B = l.Wi2; a.ldb = c->H; a.bias = l.bi2; a.out = c->d_I; a.ld_out = c->ldx;
+    a.Nout = c->N; a.K = c->H;
+    k_gemm_fma<kEpiAffine><<<dim3(ceil_div(a.Nout, kEmitTN), ceil_div(count, kEmitTM)), kEmitThreads, 0, c->stream>>>(a);
+    a.A = c->d_I; a.lda = c->ldx; a.B = l.Wj1; a.ldb = l.ldn; a.bias = l.bj1; a.out = c->d_r; a.ld_out = c->H;
+    a.Nout = c->H; a.K = c->ldx;                                   // the padding columns of both operands are zero
+    k_gemm_fma<kEpiRelu><<<dim3(ceil_div(a.Nout, kEmitTN), ceil_div(count, kEmitTM)), kEmitThreads, 0, c->stream>>>(a);
+    a.A = c->d_r; a.lda = c->H; a.B = l.Wj2; a.ldb = c->H; a.bias = l.bj2; a.add = c->d_I; a.out = c->d_x; a.ld_out = c->ldx;
+    a.Nout = c->N; a.K = c->H;
+    k_gemm_fma<kEpiScaleNoise><<<dim3(ceil_div(a.Nout, kEmitTN), ceil_div(count, kEmitTM)), kEmitThreads, 0, c->stream>>>(a);
+    c->launches += 3;
+}
+
 void launch_emission(cutoff_ctx* c, uint32_t sample_base, int count) {
+    if (c->literal) { launch_emission_literal(c, sample_base, count); return; }
     if (c->use_tc) { launch_emission_tc(c, sample_base, count); return; }
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     dim3 grid(ceil_div(c->N, kEmitTN), ceil_div(count, kEmitTM));
@@ -462,6 +555,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     c->ldx = (c->N + 7) & ~7;
     c->P = next_pow2(c->N) < 32 ? 32 : next_pow2(c->N);
     c->stream = static_cast<cudaStream_t>(cfg->stream);
+    c->literal = (cfg->flags & CUTOFF_FLAG_LITERAL) != 0;
 
     auto fail = [&](int rc) { free_all(c); delete c; return rc; };
 #define CREATE_CHECK(call)                                                                         \
@@ -483,22 +577,30 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
 
     // Pass buffers hold up to 2 GiB of samples; by default one pass covers all S samples.
     {
-        int64_t cap = (2ll << 30) / (static_cast<int64_t>(c->ldx + c->H) * sizeof(float));
+        int64_t cap = (2ll << 30) / (static_cast<int64_t>(c->ldx + c->H) * (c->literal ? 2 : 1) * sizeof(float));
         if (cap < 1024) cap = 1024;
         c->alloc_rows = cap < c->S ? static_cast<int>(cap) : c->S;
     }
     if (ceil_div(c->S, kMaxChunks) > c->alloc_rows) return fail(CUTOFF_ERR_UNSUPPORTED);   // S too large for the pass buffers
     plan_chunks(c, c->alloc_rows);
     c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
-    c->chain_tc = c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
+    c->chain_tc = !c->literal && c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
                   tc::chain_tc_smem_bytes(c->H, c->W) <= 227 * 1024;
-    c->chain_tc32 = c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
+    c->chain_tc32 = !c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
                     (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W) <= 227 * 1024;
 
     size_t blob_floats = 0;
-    for (const auto& t : tensor_specs(c->N, c->D, c->H)) blob_floats += t.rows * t.cols;
+    for (const auto& t : c->literal ? tensor_specs_literal(c->N, c->D, c->H) : tensor_specs(c->N, c->D, c->H))
+        blob_floats += (t.rows * t.cols + 7) / 8 * 8;            // each tensor starts on a 32-byte boundary
     CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
-    CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 3 * c->H * c->D));
+    CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 4 * c->H * c->D));
+    if (c->literal) {
+        CREATE_CHECK(cudaMalloc(&c->d_I, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
+        CREATE_CHECK(cudaMalloc(&c->d_r, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->H));
+        CREATE_CHECK(cudaMalloc(&c->d_Wj1p, sizeof(float) * static_cast<size_t>(c->H) * c->ldx));
+        // the padding columns of I are never written and must read as zero
+        CREATE_CHECK(cudaMemsetAsync(c->d_I, 0, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx, c->stream));
+    }
     CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     if (c->chain_tc32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H)));
@@ -517,7 +619,12 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_E, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_omega, sizeof(float) * c->N));
     if (c->use_tc) {
-        const int rc = make_tile_map(c, &c->map_v, c->d_v, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
+        int rc = make_tile_map(c, &c->map_v, c->d_v, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
+        if (!rc && c->literal)
+            rc = make_tile_map(c, &c->map_I, c->d_I, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->N),
+                               static_cast<uint64_t>(c->ldx));
+        if (!rc && c->literal)
+            rc = make_tile_map(c, &c->map_r, c->d_r, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
         if (rc) return fail(rc);
     }
     CREATE_CHECK(cudaMallocHost(&c->h_stage, sizeof(float) * c->N));
@@ -545,9 +652,9 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     std::memcpy(hdr, blob, sizeof(hdr));
     if (hdr[0] != kBlobMagic || hdr[1] != 1u) return CUTOFF_ERR_BAD_BLOB;
     if (hdr[2] != static_cast<uint32_t>(c->N) || hdr[3] != static_cast<uint32_t>(c->D) ||
-        hdr[4] != static_cast<uint32_t>(c->H))
+        hdr[4] != static_cast<uint32_t>(c->H) || hdr[5] != (c->literal ? 1u : 0u))
         return CUTOFF_ERR_BAD_BLOB;
-    const auto specs = tensor_specs(c->N, c->D, c->H);
+    const auto specs = c->literal ? tensor_specs_literal(c->N, c->D, c->H) : tensor_specs(c->N, c->D, c->H);
     size_t total = 0;
     for (const auto& t : specs) total += t.rows * t.cols;
     if (nbytes != sizeof(hdr) + total * sizeof(float)) return CUTOFF_ERR_BAD_BLOB;
@@ -557,28 +664,42 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
 
     CU_CHECK(c, cudaSetDevice(c->cfg.device));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
-    std::vector<float> host(src, src + total);
+    // device layout: every tensor starts on a 32-byte boundary (16-byte loads and tensor maps need aligned bases)
     std::vector<size_t> off(specs.size());
     size_t o = 0;
-    for (size_t i = 0; i < specs.size(); ++i) { off[i] = o; o += specs[i].rows * specs[i].cols; }
-    if (c->use_tc) {
-        // Output-layer weights as the tensor cores will see them, kept as fp32 bit patterns:
-        // bf16 (nearest even) for the bf16-weight precision, else tf32 (nearest, ties away from zero).
-        float* w4 = host.data() + off[21];
-        for (size_t i = 0; i < specs[21].rows * specs[21].cols; ++i) {
-            uint32_t u;
-            std::memcpy(&u, &w4[i], 4);
-            if (c->cfg.precision == CUTOFF_PRECISION_BF16W) u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
-            else u = (u + 0x1000u) & 0xFFFFE000u;
-            std::memcpy(&w4[i], &u, 4);
+    for (size_t i = 0; i < specs.size(); ++i) { off[i] = o; o += (specs[i].rows * specs[i].cols + 7) / 8 * 8; }
+    std::vector<float> host(o, 0.0f);
+    {
+        size_t so = 0;
+        for (size_t i = 0; i < specs.size(); ++i) {
+            const size_t n = specs[i].rows * specs[i].cols;
+            std::memcpy(host.data() + off[i], src + so, n * sizeof(float));
+            so += n;
         }
     }
-    CU_CHECK(c, cudaMemcpy(c->d_blob, host.data(), total * sizeof(float), cudaMemcpyHostToDevice));
-    // transposed copies [D][H] of the three latent-to-hidden matrices for the per-sample chain
+    if (c->use_tc) {
+        // Weights of the products that run on the tensor cores, as the tensor cores will see them, kept as
+        // fp32 bit patterns: bf16 (nearest even) for the bf16-weight precision, else tf32 (nearest, ties
+        // away from zero).  Compact variant: W4; literal variant: Wi2, Wj1, Wj2.
+        const std::vector<size_t> rounded = c->literal ? std::vector<size_t>{29, 31, 33} : std::vector<size_t>{21};
+        for (size_t t : rounded) {
+            float* wt = host.data() + off[t];
+            for (size_t i = 0; i < specs[t].rows * specs[t].cols; ++i) {
+                uint32_t u;
+                std::memcpy(&u, &wt[i], 4);
+                if (c->cfg.precision == CUTOFF_PRECISION_BF16W) u = (u + 0x7FFFu + ((u >> 16) & 1u)) & 0xFFFF0000u;
+                else u = (u + 0x1000u) & 0xFFFFE000u;
+                std::memcpy(&wt[i], &u, 4);
+            }
+        }
+    }
+    CU_CHECK(c, cudaMemcpy(c->d_blob, host.data(), host.size() * sizeof(float), cudaMemcpyHostToDevice));
+    // transposed copies [D][H] of the latent-to-hidden matrices for the per-sample chain
     const size_t D = c->D, H = c->H;
-    std::vector<float> wT(3 * H * D);
-    const size_t src_off[3] = {off[8], off[15], off[19]};           // Wz, W1, W3: each [H][D]
-    for (int t = 0; t < 3; ++t) {
+    const int n_transposed = c->literal ? 4 : 3;
+    std::vector<float> wT(n_transposed * H * D);
+    const size_t src_off[4] = {off[8], off[15], off[19], c->literal ? off[27] : 0};   // Wz, W1 | Wg1, W3 | Wh1, - | Wi1
+    for (int t = 0; t < n_transposed; ++t) {
         const float* w = host.data() + src_off[t];
         for (size_t i = 0; i < H; ++i)
             for (size_t d = 0; d < D; ++d) wT[t * H * D + d * H + i] = w[i * D + d];
@@ -679,6 +800,31 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     m.Wxb = b + off[4]; m.Whb = b + off[5]; m.bb = b + off[6]; m.b0 = b + off[7];
     m.WzT = c->d_WT; m.bz = b + off[9]; m.Wmu = b + off[10]; m.bmu = b + off[11];
     m.Wsig = b + off[12]; m.bsig = b + off[13]; m.z0 = b + off[14];
+    if (c->literal) {
+        // Wj1 [H][N] with rows padded with zeros to ldx floats (rows then start on 32 bytes for any N)
+        std::vector<float> wj1p(H * static_cast<size_t>(c->ldx), 0.0f);
+        for (size_t i = 0; i < H; ++i)
+            std::memcpy(wj1p.data() + i * c->ldx, host.data() + off[31] + i * c->N, sizeof(float) * c->N);
+        CU_CHECK(c, cudaMemcpy(c->d_Wj1p, wj1p.data(), wj1p.size() * sizeof(float), cudaMemcpyHostToDevice));
+        LiteralDev& l = c->lit;
+        l.Wg1T = c->d_WT + H * D; l.bg1 = b + off[16]; l.Wg2 = b + off[17]; l.bg2 = b + off[18];
+        l.Wh1T = c->d_WT + 2 * H * D; l.bh1 = b + off[20]; l.Wh2 = b + off[21]; l.bh2 = b + off[22];
+        l.Wl = b + off[23]; l.bl = b + off[24]; l.Ws = b + off[25]; l.bs = b + off[26];
+        l.Wi1T = c->d_WT + 3 * H * D; l.bi1 = b + off[28];
+        l.Wi2 = b + off[29]; l.bi2 = b + off[30];
+        l.Wj1 = c->d_Wj1p; l.bj1 = b + off[32]; l.ldn = c->ldx;
+        l.Wj2 = b + off[33]; l.bj2 = b + off[34];
+        m.W1T = m.b1 = m.W2 = m.b2 = m.W3T = m.b3 = m.W4 = m.b4 = nullptr;
+        if (c->use_tc) {
+            int rc = make_tile_map(c, &c->map_wi2, l.Wi2, static_cast<uint64_t>(c->N), static_cast<uint64_t>(c->H));
+            if (!rc) rc = make_tile_map(c, &c->map_wj1, l.Wj1, static_cast<uint64_t>(c->H), static_cast<uint64_t>(c->N),
+                                        static_cast<uint64_t>(c->ldx));
+            if (!rc) rc = make_tile_map(c, &c->map_wj2, l.Wj2, static_cast<uint64_t>(c->N), static_cast<uint64_t>(c->H));
+            if (rc) return rc;
+        }
+        c->weights_loaded = true;
+        return CUTOFF_OK;
+    }
     m.W1T = c->d_WT + H * D; m.b1 = b + off[16]; m.W2 = b + off[17]; m.b2 = b + off[18];
     m.W3T = c->d_WT + 2 * H * D; m.b3 = b + off[20]; m.W4 = b + off[21]; m.b4 = b + off[22];
     if (c->use_tc) {

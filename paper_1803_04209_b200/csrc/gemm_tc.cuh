@@ -1,0 +1,255 @@
+// C = A B^T with an epilogue on the 5th-generation tensor cores (tcgen05, kind::tf32): the three
+// matrix products of the literal emission of Section 3.1.3,
+//   I = u Wi2^T + bi2        r = relu(I Wj1^T + bj1)        x = I + softplus(r Wj2^T + bj2) * eps.
+//
+// Same pipeline as the emission kernel of emit_tc.cuh: one persistent CTA per SM walks over output
+// tiles of 128 rows x 256 columns; a tile is one accumulator of 128 TMEM lanes x 256 fp32 columns,
+// filled by UMMA instructions of shape M=128, N=256, K=8; operands arrive by plain per-CTA TMA loads
+// (boxes of 128 rows x 32 tf32, 128-byte swizzle; rows or columns outside the matrices read as zero)
+// into a 4-stage ring; the accumulator is double-buffered.  Warp 0 loads, warp 1 issues the MMAs,
+// warps 2..17 are the epilogue (warp w reads TMEM lanes 32*(w%4).. and the columns
+// 32*cg .. 32*cg+31 and 128+32*cg .. 128+32*cg+31 of the tile, cg = (w-2)/4).
+// Every mbarrier wait is bounded, as in emit_tc.cuh.
+#pragma once
+#include "chain_tc.cuh"      // softplus_fast
+#include "emit_tc.cuh"
+#include "kernels_literal.cuh"
+
+namespace cutoff {
+namespace tc {
+
+constexpr int kGemmBN = 256;              // output columns per tile
+
+struct GemmTcArgs {
+    const float* bias;      // [Nout]
+    const float* add;       // [M][ld_out], kEpiScaleNoise only
+    float* out;             // [M][ld_out]
+    DevState* st;
+    NoiseKey key;
+    uint32_t sample_base;
+    int M, Nout, K, ld_out;
+    int round_out;          // kEpiRelu: round the result to tf32 (it is the next product's operand)
+};
+
+template <int EPI>
+__device__ __forceinline__ void gemm_epilogue_tile(const GemmTcArgs& a, uint32_t tmem_base, uint32_t acc, int q, int cg,
+                                                   int lane, int m0, int w0, uint32_t step, uint32_t bar_acc_empty,
+                                                   const float* bias_s) {
+    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + cg * 32;
+    const int row = m0 + q * 32 + lane;
+    const bool row_ok = row < a.M;
+    const uint32_t sample = a.sample_base + static_cast<uint32_t>(row);
+    const bool wide_store = (a.ld_out & 7) == 0;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t bits[2][16];
+        tmem_ld16(taddr + 16 * half, bits[0]);
+        tmem_ld16(taddr + 128 + 16 * half, bits[1]);
+        tmem_ld_wait();
+        if (half == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * acc);    // accumulator is free again
+        }
+#pragma unroll
+        for (int part = 0; part < 2; ++part) {
+            const int jw = w0 + 128 * part + cg * 32 + 16 * half;
+            if (!row_ok || jw >= a.Nout) continue;
+            float* dst = a.out + static_cast<size_t>(row) * a.ld_out + jw;
+            float out[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int j = jw + 4 * i;
+                if (j >= a.Nout) continue;
+                const float4 bv = *reinterpret_cast<const float4*>(bias_s + 32 * part + 16 * half + 4 * i);
+                const float b[4] = {bv.x, bv.y, bv.z, bv.w};
+                float eps[4] = {0.f, 0.f, 0.f, 0.f}, base[4] = {0.f, 0.f, 0.f, 0.f};
+                if (EPI == kEpiScaleNoise) {
+                    normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
+                                 a.key.seed_hi, eps);
+                    const float4 iv = *reinterpret_cast<const float4*>(a.add + static_cast<size_t>(row) * a.ld_out + j);
+                    base[0] = iv.x; base[1] = iv.y; base[2] = iv.z; base[3] = iv.w;
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float v = __uint_as_float(bits[part][4 * i + c]) + b[c];
+                    if (EPI == kEpiRelu) {
+                        v = fmaxf(v, 0.0f);
+                        if (a.round_out) v = round_tf32(v);
+                    }
+                    if (EPI == kEpiScaleNoise) v = fmaf(softplus_fast(v), eps[c], base[c]);
+                    out[4 * i + c] = v;
+                }
+            }
+#pragma unroll
+            for (int p = 0; p < 2; ++p) {
+                if (wide_store && jw + 8 * p + 7 < a.Nout) {
+                    store8(dst + 8 * p, out + 8 * p);
+                    continue;
+                }
+#pragma unroll
+                for (int i = 2 * p; i < 2 * p + 2; ++i) {
+                    const int ji = jw + 4 * i;
+                    if (ji + 3 < a.Nout) {
+                        *reinterpret_cast<float4*>(dst + 4 * i) =
+                            make_float4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
+                    } else {
+                        for (int c = 0; c < 4 && ji + c < a.Nout; ++c) dst[4 * i + c] = out[4 * i + c];
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(kThreads, 1) k_gemm_tc(const __grid_constant__ CUtensorMap map_a,
+                                                          const __grid_constant__ CUtensorMap map_b, GemmTcArgs a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;                     // operand ring, 1024-byte aligned
+    const uint32_t bars = tiles + kStages * kStageBytes;
+    // barrier layout (8 bytes each): full[4], empty[4], acc_full[2], acc_empty[2], drain; then tmem base, abort flag
+    const uint32_t bar_full = bars, bar_empty = bars + 8 * kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * kStages, bar_acc_empty = bar_acc_full + 16;
+    const uint32_t bar_drain = bar_acc_empty + 16;
+    uint8_t* gen = smem_raw + (tiles - raw) + kStages * kStageBytes;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(gen + 8 * (2 * kStages + 5));
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen + 8 * (2 * kStages + 5) + 8);
+    float* bias_all = reinterpret_cast<float*>(gen + 256);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_tiles_w = ceil_div(a.Nout, kGemmBN);
+    const int n_tiles_m = ceil_div(a.M, kBM);
+    const int total_tiles = n_tiles_w * n_tiles_m;
+    const int k_blocks = ceil_div(a.K, kBK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bar_acc_full + 8 * b, 1);
+            mbar_init(bar_acc_empty + 8 * b, kEpiWarps);
+        }
+        mbar_init(bar_drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------------------------------------------------
+        uint32_t stage = 0, phase = 0;
+        uint32_t armed_mask = 0, parity_mask = 0;      // per stage: armed at least once / parity of its last phase
+        bool ok = true;
+        for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+            const int m0 = (t / n_tiles_w) * kBM, w0 = (t % n_tiles_w) * kGemmBN;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abort_flag, a.st);
+                if (!ok) break;
+                if (lane == 0) {
+                    const uint32_t full = bar_full + 8 * stage;
+                    const uint32_t dst = tiles + stage * kStageBytes;
+                    mbar_arrive_expect_tx(full, kStageBytes);
+                    tma_load_2d(dst, &map_a, kb * kBK, m0, full);
+                    tma_load_2d(dst + kABytes, &map_b, kb * kBK, w0, full);
+                    tma_load_2d(dst + kABytes + kBBytes / 2, &map_b, kb * kBK, w0 + 128, full);
+                }
+                __syncwarp();
+                armed_mask |= 1u << stage;
+                parity_mask = (parity_mask & ~(1u << stage)) | (phase << stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok) {
+            // wind down: let every copy that was issued land before the CTA leaves (bounded)
+            for (uint32_t s = 0; s < static_cast<uint32_t>(kStages); ++s) {
+                if (!((armed_mask >> s) & 1u)) continue;
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bar_full + 8 * s, (parity_mask >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer -------------------------------------------------------------
+        uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+            ok = mbar_wait(bar_acc_empty + 8 * acc, acc_phase ^ 1u, abort_flag, a.st);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + acc * kAccCols;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                ok = mbar_wait(bar_full + 8 * stage, phase, abort_flag, a.st);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    const uint32_t a_addr = tiles + stage * kStageBytes;
+                    const uint64_t a_desc = make_smem_desc(a_addr);
+                    const uint64_t b_desc = make_smem_desc(a_addr + kABytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 8; ++k)          // 8 tf32 = 32 bytes per instruction
+                        umma_tf32(d_tmem, a_desc + 2 * k, b_desc + 2 * k, kInstrDesc, (kb | k) != 0);
+                    umma_commit(bar_empty + 8 * stage);         // frees the stage when these MMAs are done
+                    if (kb == k_blocks - 1) umma_commit(bar_acc_full + 8 * acc);
+                }
+                __syncwarp();
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (!ok) {
+            // make sure no MMA is still running before TMEM is released (bounded)
+            if (lane == 0) umma_commit(bar_drain);
+            __syncwarp();
+            const unsigned long long t0 = global_ns();
+            while (!mbar_try_wait(bar_drain, 0u) && global_ns() - t0 < kWaitLimitNs) {}
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue ---------------------------------------------------------------
+        const int q = warp & 3, cg = (warp - 2) >> 2;
+        const uint32_t step = EPI == kEpiScaleNoise ? a.st->step : 0u;
+        float* bias_s = bias_all + (warp - 2) * 64;
+        int w_staged = -1;
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; ok && t < total_tiles; t += gridDim.x) {
+            const int m0 = (t / n_tiles_w) * kBM, w0 = (t % n_tiles_w) * kGemmBN;
+            if (w0 != w_staged) {                       // biases of this warp's 2 x 32 columns, read once per column tile
+                const int j = w0 + cg * 32 + lane;
+                const float b_lo = j < a.Nout ? __ldg(a.bias + j) : 0.f;
+                const float b_hi = j + 128 < a.Nout ? __ldg(a.bias + j + 128) : 0.f;
+                __syncwarp();                           // the previous tile's readers are done
+                bias_s[lane] = b_lo;
+                bias_s[32 + lane] = b_hi;
+                __syncwarp();
+                w_staged = w0;
+            }
+            ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, a.st);
+            if (!ok) break;
+            tc_fence_after();
+            gemm_epilogue_tile<EPI>(a, tmem_base, acc, q, cg, lane, m0, w0, step, bar_acc_empty, bias_s);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+}  // namespace tc
+}  // namespace cutoff

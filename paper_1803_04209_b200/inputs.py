@@ -117,7 +117,7 @@ def make_weights(N: int, D: int, H: int, seed: int = 0, std: float = 0.1,
 
 
 def make_weights_literal(N: int, D: int, H: int, seed: int = 0, std: float = 0.1,
-                         fan_in_ref: int | None = None, offsets: bool = True) -> dict:
+                         fan_in_ref: int | None = None, offsets: bool = True, bf16: bool = False) -> dict:
     """Random-initialised weights of the literal variant, drawn like `make_weights`.
 
     ``offsets=True`` moves the untrained model into the regime of a fitted one:
@@ -140,6 +140,8 @@ def make_weights_literal(N: int, D: int, H: int, seed: int = 0, std: float = 0.1
         w["bi2"] = w["bi2"] * np.float32(0.5) + np.float32(0.5)
         w["bj2"] += np.float32(math.log(math.expm1(0.05)))
         w["bs"] += np.float32(math.log(math.expm1(0.1)))
+    if bf16:
+        w = {k: round_to_bf16(v) for k, v in w.items()}
     return w
 
 
@@ -187,7 +189,8 @@ WORKLOADS = {
 
 
 def workload_weights_literal(wl: Workload, offsets: bool = True) -> dict:
-    return make_weights_literal(wl.N, wl.D, wl.H, seed=wl.weight_seed, std=0.1, fan_in_ref=32, offsets=offsets)
+    return make_weights_literal(wl.N, wl.D, wl.H, seed=wl.weight_seed, std=0.1, fan_in_ref=32, offsets=offsets,
+                                bf16=(wl.precision == 2))
 
 
 def workload_weights(wl: Workload, offsets: bool = True) -> dict:
