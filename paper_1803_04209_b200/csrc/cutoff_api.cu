@@ -178,7 +178,7 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
     // CTAs of the sort kernel per pass: enough to fill the GPU, within the partial-sum rows available
     int want, cap;
     if (c->P <= 1024) { want = ceil_div(rows, kSortWarps); cap = c->sm_count * 2; }
-    else { want = rows; cap = c->sm_count * (c->P == 2048 ? 8 : 4); }
+    else { want = rows; cap = c->sm_count * 8; }
     if (cap > kPartialRows / c->n_chunks) cap = kPartialRows / c->n_chunks;
     c->sort_grid = want < cap ? want : cap;
 }

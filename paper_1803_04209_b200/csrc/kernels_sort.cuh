@@ -47,92 +47,14 @@ template <> struct KeyOps<unsigned long long> {
 // below E stay inside a lane's registers (one min and one max per pair); distances of E and more
 // are lane exchanges by shuffle in the reversed-key form described above (one min per key; the
 // reversals are multiplications by +-1, which run on the otherwise idle FMA pipe).
+// The register stages are always unrolled (their register indices must be static); the merges across
+// lanes are unrolled too, or (LOOPED) a run-time loop over the merge width.
 // Ascending on exit.
-template <typename T, int E>
-__device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
-    using Ops = KeyOps<T>;
-    typename Ops::Flip cur = Ops::identity();             // form the lane's keys are held in
-#pragma unroll
-    for (int k = 2; k <= 32 * E; k <<= 1) {
-        if (k <= E) {
-#pragma unroll
-            for (int r = 0; r < E; ++r) {
-                const int p = r ^ (k - 1);
-                if (p > r) {
-                    const T a = v[r], b = v[p];
-                    v[r] = Ops::lo(a, b);
-                    v[p] = Ops::hi(a, b);
-                }
-            }
-        } else {
-            const int lane_mask = k / E - 1;
-            const typename Ops::Flip want = Ops::flip_if((lane & (k / (2 * E))) != 0);
-            const typename Ops::Flip f = Ops::combine(want, cur);
-            cur = want;
-#pragma unroll
-            for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
-            T other[E];
-#pragma unroll
-            for (int r = 0; r < E; ++r) other[r] = Ops::shfl_xor(v[E - 1 - r], lane_mask);
-#pragma unroll
-            for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], Ops::reverse(other[r]));
-        }
-#pragma unroll
-        for (int j = k >> 2; j > 0; j >>= 1) {
-            if (j < E) {
-                if (k > E && j == E / 2) {                // back to plain keys before the register stages
-#pragma unroll
-                    for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
-                    cur = Ops::identity();
-                }
-#pragma unroll
-                for (int r = 0; r < E; ++r) {
-                    if ((r & j) == 0) {
-                        const T a = v[r], b = v[r | j];
-                        v[r] = Ops::lo(a, b);
-                        v[r | j] = Ops::hi(a, b);
-                    }
-                }
-            } else {
-                const int lane_mask = j / E;
-                const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
-                const typename Ops::Flip f = Ops::combine(want, cur);
-                cur = want;
-#pragma unroll
-                for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
-#pragma unroll
-                for (int r = 0; r < E; ++r) {
-                    const T other = Ops::shfl_xor(v[r], lane_mask);
-                    v[r] = Ops::lo(v[r], Ops::reverse(other));
-                }
-            }
-        }
-    }
-    if (E == 1) v[0] = Ops::apply(v[0], cur);             // no register stage ever undid the reversal
-}
 
-// The half-cleaners idx <-> idx ^ j for j = 16E .. 1 of one merge, inside a warp: what remains of a
-// merge wider than the warp once its cross-warp exchanges are done.  Plain keys in, plain keys out.
+// Half-cleaners idx <-> idx ^ j for j = E/2 .. 1: inside a lane's registers.
 template <typename T, int E>
-__device__ __forceinline__ void warp_half_cleaners(T (&v)[E], int lane) {
+__device__ __forceinline__ void lane_half_cleaners(T (&v)[E]) {
     using Ops = KeyOps<T>;
-    typename Ops::Flip cur = Ops::identity();
-#pragma unroll
-    for (int j = 16 * E; j >= E; j >>= 1) {
-        const int lane_mask = j / E;
-        const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
-        const typename Ops::Flip f = Ops::combine(want, cur);
-        cur = want;
-#pragma unroll
-        for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
-#pragma unroll
-        for (int r = 0; r < E; ++r) {
-            const T other = Ops::shfl_xor(v[r], lane_mask);
-            v[r] = Ops::lo(v[r], Ops::reverse(other));
-        }
-    }
-#pragma unroll
-    for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
 #pragma unroll
     for (int j = E / 2; j > 0; j >>= 1) {
 #pragma unroll
@@ -146,6 +68,112 @@ __device__ __forceinline__ void warp_half_cleaners(T (&v)[E], int lane) {
     }
 }
 
+// Half-cleaners between lanes, lane distances first_mask, first_mask/2, .. 1, in the reversed-key form.
+// `cur` is the form the lane's keys are held in on entry; plain keys on exit.
+template <typename T, int E>
+__device__ __forceinline__ void shuffle_half_cleaners(T (&v)[E], int lane, int first_mask, typename KeyOps<T>::Flip cur) {
+    using Ops = KeyOps<T>;
+#pragma unroll 1
+    for (int lane_mask = first_mask; lane_mask > 0; lane_mask >>= 1) {
+        const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
+        const typename Ops::Flip f = Ops::combine(want, cur);
+        cur = want;
+#pragma unroll
+        for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const T other = Ops::shfl_xor(v[r], lane_mask);
+            v[r] = Ops::lo(v[r], Ops::reverse(other));
+        }
+    }
+#pragma unroll
+    for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+}
+
+template <typename T, int E, bool LOOPED = false>
+__device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
+    using Ops = KeyOps<T>;
+    // merges of width 2 .. E: each lane sorts its own keys
+#pragma unroll
+    for (int k = 2; k <= E; k <<= 1) {
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int p = r ^ (k - 1);
+            if (p > r) {
+                const T a = v[r], b = v[p];
+                v[r] = Ops::lo(a, b);
+                v[p] = Ops::hi(a, b);
+            }
+        }
+#pragma unroll
+        for (int j = k >> 2; j > 0; j >>= 1) {
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                if ((r & j) == 0) {
+                    const T a = v[r], b = v[r | j];
+                    v[r] = Ops::lo(a, b);
+                    v[r | j] = Ops::hi(a, b);
+                }
+            }
+        }
+    }
+    if (!LOOPED) {
+        // merges of width 2E .. 32E, m = lanes per merge, fully unrolled: the fastest form when one warp sorts a row
+#pragma unroll
+        for (int m = 2; m <= 32; m <<= 1) {
+            typename Ops::Flip cur = Ops::flip_if((lane & (m >> 1)) != 0);
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+            T other[E];
+#pragma unroll
+            for (int r = 0; r < E; ++r) other[r] = Ops::shfl_xor(v[E - 1 - r], m - 1);
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], Ops::reverse(other[r]));
+#pragma unroll
+            for (int lane_mask = m >> 2; lane_mask > 0; lane_mask >>= 1) {
+                const typename Ops::Flip want = Ops::flip_if((lane & lane_mask) != 0);
+                const typename Ops::Flip f = Ops::combine(want, cur);
+                cur = want;
+#pragma unroll
+                for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], f);
+#pragma unroll
+                for (int r = 0; r < E; ++r) {
+                    const T o = Ops::shfl_xor(v[r], lane_mask);
+                    v[r] = Ops::lo(v[r], Ops::reverse(o));
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+            lane_half_cleaners<T, E>(v);
+        }
+        return;
+    }
+    // the same merges as a run-time loop whose body serves all five widths: a fraction of the code, for the
+    // kernels in which several warps share a row (unrolled, their code overflows the instruction cache)
+#pragma unroll 1
+    for (int m = 2; m <= 32; m <<= 1) {
+        // mirror exchange idx <-> idx ^ (mE - 1): lane ^ (m-1), register E-1-r
+        const typename Ops::Flip cur = Ops::flip_if((lane & (m >> 1)) != 0);
+#pragma unroll
+        for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
+        T other[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) other[r] = Ops::shfl_xor(v[E - 1 - r], m - 1);
+#pragma unroll
+        for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], Ops::reverse(other[r]));
+        shuffle_half_cleaners<T, E>(v, lane, m >> 2, cur);
+        lane_half_cleaners<T, E>(v);
+    }
+}
+
+// The half-cleaners idx <-> idx ^ j for j = 16E .. 1 of one merge, inside a warp: what remains of a
+// merge wider than the warp once its cross-warp exchanges are done.  Plain keys in, plain keys out.
+template <typename T, int E>
+__device__ __forceinline__ void warp_half_cleaners(T (&v)[E], int lane) {
+    shuffle_half_cleaners<T, E>(v, lane, 16, KeyOps<T>::identity());
+    lane_half_cleaners<T, E>(v);
+}
+
 // Bitonic sorting network over WPR * 1024 keys held by the WPR warps of a CTA, 32 keys per lane,
 // key index idx = (warp * 32 + lane) * 32 + r.  Each warp first sorts its 1024 keys in registers
 // and by shuffles; the merges of width 2048 and 4096 then start with exchanges between warps (one
@@ -157,8 +185,8 @@ __device__ __forceinline__ void cta_bitonic_sort(T (&v)[32], T* xch) {
     using Ops = KeyOps<T>;
     constexpr int E = 32, T_ = WPR * 32;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    warp_bitonic_sort<T, E>(v, lane);
-#pragma unroll
+    warp_bitonic_sort<T, E, true>(v, lane);
+#pragma unroll 1
     for (int k = 2; k <= WPR; k <<= 1) {                 // merge width in warps
         // mirror exchange: idx <-> idx ^ (k*1024 - 1)
         {
@@ -176,7 +204,7 @@ __device__ __forceinline__ void cta_bitonic_sort(T (&v)[32], T* xch) {
             __syncthreads();
         }
         // half-cleaners between warps: idx <-> idx ^ (j*1024), j = k/4 .. 1
-#pragma unroll
+#pragma unroll 1
         for (int j = k >> 2; j > 0; j >>= 1) {
 #pragma unroll
             for (int r = 0; r < E; ++r) xch[r * T_ + threadIdx.x] = v[r];
@@ -351,7 +379,7 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
 // registers, running sums in registers, one partial row per CTA.
 // ---------------------------------------------------------------------------------------------
 template <int WPR, bool SQ>
-__global__ void __launch_bounds__(WPR * 32) k_sort_sum_cta(const float* __restrict__ x, int ldx, int N, int count,
+__global__ void __launch_bounds__(WPR * 32, SQ ? 3 : 4) k_sort_sum_cta(const float* __restrict__ x, int ldx, int N, int count,
                                                             float* __restrict__ partial, float* __restrict__ partial_sq) {
     __shared__ float xch[WPR * 1024];
     constexpr int E = 32, T_ = WPR * 32;
