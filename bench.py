@@ -42,10 +42,24 @@ NCU_TRAFFIC = {
 PRECISION_NAMES = {0: "f32", 1: "tf32", 2: "tf32(bf16 weights)"}
 
 
+def odd_even_merge_sort_size(n: int) -> int:
+    """Compare-exchanges of Batcher's odd-even merge sort over n = 2^k keys."""
+    def merge(n, r):
+        return 2 * merge(n, 2 * r) + (n // (2 * r) - 1) if 2 * r < n else 1
+    return 0 if n < 2 else 2 * odd_even_merge_sort_size(n // 2) + merge(n, 1)
+
+
 def compare_exchanges(n_pow2: int) -> int:
-    """Compare-exchange operations of a bitonic network over n_pow2 keys."""
-    lg = n_pow2.bit_length() - 1
-    return (n_pow2 // 2) * lg * (lg + 1) // 2
+    """Compare-exchanges of the library's network over n_pow2 keys: every lane sorts its E = min(32, n/32) keys
+    by odd-even merge sort, then bitonic merges of width 2E .. n (n/2 compare-exchanges per stage, log2(k)
+    stages for width k)."""
+    e = min(32, n_pow2 // 32)
+    total = (n_pow2 // e) * odd_even_merge_sort_size(e)
+    k = 2 * e
+    while k <= n_pow2:
+        total += (n_pow2 // 2) * (k.bit_length() - 1)
+        k *= 2
+    return total
 
 
 def stage_work(wl, S, literal=False):

@@ -40,8 +40,9 @@ template <> struct KeyOps<unsigned long long> {
     static __device__ __forceinline__ T reverse(T v) { return ~v; }
 };
 
-// Bitonic sorting network over 32*E keys held by one warp, E keys per lane, key index
-// idx = lane*E + r ("blocked").  Every merge of width k starts with the mirror exchange
+// Sorting network over 32*E keys held by one warp, E keys per lane, key index idx = lane*E + r
+// ("blocked"): every lane first sorts its own keys (lane_sort), then bitonic merges of width
+// k = 2E .. 32E combine them.  Every merge of width k starts with the mirror exchange
 // idx <-> idx ^ (k-1) and continues with half-cleaners idx <-> idx ^ j, j = k/4 .. 1; the lower
 // index always keeps the smaller key, so no exchange depends on a direction flag.  Distances
 // below E stay inside a lane's registers (one min and one max per pair); distances of E and more
@@ -65,6 +66,37 @@ __device__ __forceinline__ void lane_half_cleaners(T (&v)[E]) {
                 v[r | j] = Ops::hi(a, b);
             }
         }
+    }
+}
+
+// A lane's own E keys, ascending: Batcher's odd-even merge sort (Batcher, "Sorting networks and their
+// applications", 1968), which needs fewer compare-exchanges than the bitonic network (191 against 240 for
+// 32 keys) at the same depth.  All indices are compile-time constants, so the keys stay in registers.
+template <typename T, int E, int LO, int N, int R>
+__device__ __forceinline__ void lane_odd_even_merge(T (&v)[E]) {
+    using Ops = KeyOps<T>;
+    constexpr int M = 2 * R;
+    if constexpr (M < N) {
+        lane_odd_even_merge<T, E, LO, N, M>(v);          // even subsequence
+        lane_odd_even_merge<T, E, LO + R, N, M>(v);      // odd subsequence
+#pragma unroll
+        for (int i = LO + R; i + R < LO + N; i += M) {
+            const T a = v[i], b = v[i + R];
+            v[i] = Ops::lo(a, b);
+            v[i + R] = Ops::hi(a, b);
+        }
+    } else {
+        const T a = v[LO], b = v[LO + R];
+        v[LO] = Ops::lo(a, b);
+        v[LO + R] = Ops::hi(a, b);
+    }
+}
+template <typename T, int E, int LO, int N>
+__device__ __forceinline__ void lane_sort(T (&v)[E]) {
+    if constexpr (N > 1) {
+        lane_sort<T, E, LO, N / 2>(v);
+        lane_sort<T, E, LO + N / 2, N / 2>(v);
+        lane_odd_even_merge<T, E, LO, N, 1>(v);
     }
 }
 
@@ -93,30 +125,7 @@ __device__ __forceinline__ void shuffle_half_cleaners(T (&v)[E], int lane, int f
 template <typename T, int E, bool LOOPED = false>
 __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
     using Ops = KeyOps<T>;
-    // merges of width 2 .. E: each lane sorts its own keys
-#pragma unroll
-    for (int k = 2; k <= E; k <<= 1) {
-#pragma unroll
-        for (int r = 0; r < E; ++r) {
-            const int p = r ^ (k - 1);
-            if (p > r) {
-                const T a = v[r], b = v[p];
-                v[r] = Ops::lo(a, b);
-                v[p] = Ops::hi(a, b);
-            }
-        }
-#pragma unroll
-        for (int j = k >> 2; j > 0; j >>= 1) {
-#pragma unroll
-            for (int r = 0; r < E; ++r) {
-                if ((r & j) == 0) {
-                    const T a = v[r], b = v[r | j];
-                    v[r] = Ops::lo(a, b);
-                    v[r | j] = Ops::hi(a, b);
-                }
-            }
-        }
-    }
+    lane_sort<T, E, 0, E>(v);                // each lane sorts its own keys
     if (!LOOPED) {
         // merges of width 2E .. 32E, m = lanes per merge, fully unrolled: the fastest form when one warp sorts a row
 #pragma unroll
