@@ -126,7 +126,7 @@ template <typename T, int E, bool LOOPED = false>
 __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
     using Ops = KeyOps<T>;
     lane_sort<T, E, 0, E>(v);                // each lane sorts its own keys
-    if (!LOOPED) {
+    if constexpr (!LOOPED) {
         // merges of width 2E .. 32E, m = lanes per merge, fully unrolled: the fastest form when one warp sorts a row
 #pragma unroll
         for (int m = 2; m <= 32; m <<= 1) {
@@ -155,8 +155,7 @@ __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
             for (int r = 0; r < E; ++r) v[r] = Ops::apply(v[r], cur);
             lane_half_cleaners<T, E>(v);
         }
-        return;
-    }
+    } else {
     // the same merges as a run-time loop whose body serves all five widths: a fraction of the code, for the
     // kernels in which several warps share a row (unrolled, their code overflows the instruction cache)
 #pragma unroll 1
@@ -172,6 +171,7 @@ __device__ __forceinline__ void warp_bitonic_sort(T (&v)[E], int lane) {
         for (int r = 0; r < E; ++r) v[r] = Ops::lo(v[r], Ops::reverse(other[r]));
         shuffle_half_cleaners<T, E>(v, lane, m >> 2, cur);
         lane_half_cleaners<T, E>(v);
+    }
     }
 }
 
