@@ -56,7 +56,8 @@ struct cutoff_ctx {
     uint8_t* h_mask = nullptr;      // pinned [N]
     bool draws_valid = false;       // d_x holds every predictive draw of the last decision (needed for imputation)
     DevState* d_state = nullptr;
-    float* d_proj = nullptr;        // [2][W][H]
+    float* d_proj = nullptr;        // [2][W slots][H] raw input projections of the ring's vectors, kept up to date by every push
+    bool proj_stale = true;         // the ring or the weights were replaced: recompute every slot before the next decision
     float* d_hlr = nullptr;         // [2][W][H]
     float* d_v = nullptr;           // [chunk_rows][H]
     float* d_x = nullptr;           // [chunk_rows][ldx]
@@ -428,12 +429,24 @@ void launch_rnn_resident(cutoff_ctx* c) {
         attr_set = true;
     }
     const size_t smem = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float);
-    k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_WhR, c->d_proj, c->d_hlr);
+    k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_WhR, c->d_proj, c->d_state, c->d_hlr);
+}
+
+// Input projections: of the newest vector after a push, of every slot when the ring or the weights changed.
+void launch_projection(cutoff_ctx* c, bool newest_only) {
+    dim3 grid(ceil_div(c->H, kProjWarps), 2);
+    k_enc_proj<<<grid, kProjWarps * 32, 0, c->stream>>>(c->m, c->d_ring, c->d_state, newest_only ? 1 : 0, c->d_proj);
+    c->launches += 1;
+}
+
+void refresh_projections(cutoff_ctx* c) {
+    if (!c->proj_stale) return;
+    launch_projection(c, false);
+    c->proj_stale = false;
 }
 
 void launch_encoder(cutoff_ctx* c) {
-    dim3 grid(ceil_div(c->H, kProjWarps), 2);
-    k_enc_proj<<<grid, kProjWarps * 32, 0, c->stream>>>(c->m, c->d_ring, c->d_state, c->d_proj);
+    refresh_projections(c);
     const bool fits = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float) <= 200 * 1024;
     switch (fits ? c->H : 0) {
         case 32: launch_rnn_resident<8>(c); break;
@@ -441,9 +454,9 @@ void launch_encoder(cutoff_ctx* c) {
         case 128: launch_rnn_resident<32>(c); break;
         case 256: launch_rnn_resident<64>(c); break;
         default:
-            k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_hlr);
+            k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
     }
-    c->launches += 2;
+    c->launches += 1;
 }
 
 int ensure_events(cutoff_ctx* c) {
@@ -823,6 +836,7 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
             if (rc) return rc;
         }
         c->weights_loaded = true;
+        c->proj_stale = true;
         return CUTOFF_OK;
     }
     m.W1T = c->d_WT + H * D; m.b1 = b + off[16]; m.W2 = b + off[17]; m.b2 = b + off[18];
@@ -832,12 +846,14 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         if (rc) return rc;
     }
     c->weights_loaded = true;
+    c->proj_stale = true;
     return CUTOFF_OK;
 }
 
 static int push_common(cutoff_ctx* c, const float* dev_src) {
     k_push<<<1, kPushThreads, 0, c->stream>>>(dev_src, c->d_ring, c->d_state, c->N, c->W);
     c->launches += 1;
+    if (c->weights_loaded && !c->proj_stale) launch_projection(c, true);     // else every slot is redone before the next decision
     CU_CHECK(c, cudaGetLastError());
     c->pushes += 1;
     return CUTOFF_OK;
@@ -967,11 +983,13 @@ int cutoff_predict(cutoff_ctx* c, int32_t* c_out) {
 // changing argument because the window position, the normaliser and the decision counter live
 // in device memory.
 static int build_graph(cutoff_ctx* c) {
+    refresh_projections(c);                        // not part of the graph: replays only project the vector they push
     const int64_t launches_before = c->launches;
     CU_CHECK(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
     cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, cudaMemcpyHostToDevice, c->stream);
     k_push<<<1, kPushThreads, 0, c->stream>>>(c->d_stage, c->d_ring, c->d_state, c->N, c->W);
     c->launches += 1;
+    launch_projection(c, true);
     const bool timing = c->timing;
     c->timing = false;
     const int rc = enqueue_decision(c);
@@ -1010,6 +1028,7 @@ int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
         if (rc) return rc;
     }
     std::memcpy(c->h_stage, runtimes_sec, sizeof(float) * c->N);     // the stream is idle: every call ends synchronised
+    refresh_projections(c);                        // after a restore or new weights; the replay then adds the new vector
     CU_CHECK(c, cudaGraphLaunch(c->graph_exec, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     c->launches += c->graph_kernels;
@@ -1077,6 +1096,7 @@ int cutoff_reset(cutoff_ctx* c) {
     c->pending = false;
     c->have_result = false;
     c->draws_valid = false;
+    c->proj_stale = true;
     return CUTOFF_OK;
 }
 
@@ -1117,6 +1137,7 @@ int cutoff_restore_state(cutoff_ctx* c, const void* buf, size_t nbytes) {
     c->pushes = s.push_count;
     c->pending = false;
     c->have_result = false;
+    c->proj_stale = true;
     return CUTOFF_OK;
 }
 

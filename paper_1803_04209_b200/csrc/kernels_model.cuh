@@ -110,33 +110,34 @@ __global__ void __launch_bounds__(kImputeThreads) k_impute(float* __restrict__ s
 }
 
 // ---------------------------------------------------------------------------------------------
-// Encoder, part 1: input projections of both RNNs for every window position,
-//   P[dir][t][i] = sum_j Wx_dir[i][j] * xhat_t[j] + b_dir[i],   xhat_t = x_t / s.
-// One warp per hidden unit i; the weight row is read once for all window positions.
-// Window position t (0 = oldest) lives in ring slot (push_count + t) mod W.
+// Encoder, part 1: input projections of both RNNs, cached per ring slot,
+//   R[dir][slot][i] = sum_j Wx_dir[i][j] * x_slot[j]          (raw seconds: the normaliser is applied by part 2,
+//                                                              so a slot's projection never has to be redone)
+// One warp per hidden unit i; the weight row is read once for all slots of the launch.
+// newest_only = 1: only the slot of the vector pushed last (launched after every push);
+// newest_only = 0: every slot (after the ring or the weights were replaced).  Both run the same
+// arithmetic per slot, so a cached projection equals a recomputed one bit for bit.
 // ---------------------------------------------------------------------------------------------
 constexpr int kProjWarps = 8;
 constexpr int kProjChunk = 8;
 
 __global__ void __launch_bounds__(kProjWarps * 32) k_enc_proj(ModelDev m, const float* __restrict__ ring,
-                                                               const DevState* __restrict__ st,
-                                                               float* __restrict__ proj /*[2][W][H]*/) {
+                                                               const DevState* __restrict__ st, int newest_only,
+                                                               float* __restrict__ proj /*[2][W slots][H]*/) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int i = blockIdx.x * kProjWarps + warp;
     const int dir = blockIdx.y;
     if (i >= m.H) return;
     const float* Wx = (dir ? m.Wxb : m.Wxf) + static_cast<size_t>(i) * m.N;
-    const float bias = (dir ? m.bb : m.bf)[i];
-    const uint32_t pushes = st->push_count;
-    const float inv_scale = st->inv_scale;
-    for (int t0 = 0; t0 < m.W; t0 += kProjChunk) {
+    const int slot_first = newest_only ? static_cast<int>((st->push_count + m.W - 1) % m.W) : 0;
+    const int n_slots = newest_only ? 1 : m.W;
+    for (int s0 = 0; s0 < n_slots; s0 += kProjChunk) {
         float acc[kProjChunk];
         const float* row[kProjChunk];
 #pragma unroll
         for (int tt = 0; tt < kProjChunk; ++tt) {
             acc[tt] = 0.0f;
-            const int t = min(t0 + tt, m.W - 1);
-            row[tt] = ring + static_cast<size_t>((pushes + t) % m.W) * m.N;
+            row[tt] = ring + static_cast<size_t>(slot_first + min(s0 + tt, n_slots - 1)) * m.N;
         }
         if ((m.N & 3) == 0) {
             // 16-byte loads, four independent iterations in flight
@@ -145,18 +146,22 @@ __global__ void __launch_bounds__(kProjWarps * 32) k_enc_proj(ModelDev m, const 
                 const float4 w = *reinterpret_cast<const float4*>(Wx + j);
 #pragma unroll
                 for (int tt = 0; tt < kProjChunk; ++tt) {
+                    if (s0 + tt >= n_slots) break;          // uniform: one slot after a push
                     const float4 xv = *reinterpret_cast<const float4*>(row[tt] + j);
-                    acc[tt] = fmaf(w.x, xv.x * inv_scale, acc[tt]);
-                    acc[tt] = fmaf(w.y, xv.y * inv_scale, acc[tt]);
-                    acc[tt] = fmaf(w.z, xv.z * inv_scale, acc[tt]);
-                    acc[tt] = fmaf(w.w, xv.w * inv_scale, acc[tt]);
+                    acc[tt] = fmaf(w.x, xv.x, acc[tt]);
+                    acc[tt] = fmaf(w.y, xv.y, acc[tt]);
+                    acc[tt] = fmaf(w.z, xv.z, acc[tt]);
+                    acc[tt] = fmaf(w.w, xv.w, acc[tt]);
                 }
             }
         } else {
             for (int j = lane; j < m.N; j += 32) {
                 const float w = Wx[j];
 #pragma unroll
-                for (int tt = 0; tt < kProjChunk; ++tt) acc[tt] = fmaf(w, row[tt][j] * inv_scale, acc[tt]);
+                for (int tt = 0; tt < kProjChunk; ++tt) {
+                    if (s0 + tt >= n_slots) break;
+                    acc[tt] = fmaf(w, row[tt][j], acc[tt]);
+                }
             }
         }
 #pragma unroll
@@ -164,9 +169,19 @@ __global__ void __launch_bounds__(kProjWarps * 32) k_enc_proj(ModelDev m, const 
             float v = acc[tt];
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-            if (lane == 0 && t0 + tt < m.W) proj[(static_cast<size_t>(dir) * m.W + t0 + tt) * m.H + i] = v + bias;
+            if (lane == 0 && s0 + tt < n_slots)
+                proj[(static_cast<size_t>(dir) * m.W + slot_first + s0 + tt) * m.H + i] = v;
         }
     }
+}
+
+// Input projection of window position t (0 = oldest) for hidden unit i: the cached raw projection of the ring slot
+// that holds position t, scaled by 1 / s (Section 3.1.3: observations are divided by twice the mean of the first
+// window), plus the bias.
+__device__ __forceinline__ float window_projection(const ModelDev& m, const float* __restrict__ proj, int dir, int t, int i,
+                                                   uint32_t pushes, float inv_scale) {
+    const int slot = static_cast<int>((pushes + static_cast<uint32_t>(t)) % static_cast<uint32_t>(m.W));
+    return fmaf(proj[(static_cast<size_t>(dir) * m.W + slot) * m.H + i], inv_scale, (dir ? m.bb : m.bf)[i]);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -177,6 +192,7 @@ __global__ void __launch_bounds__(kProjWarps * 32) k_enc_proj(ModelDev m, const 
 constexpr int kRnnThreads = 1024;
 
 __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float* __restrict__ proj,
+                                                          const DevState* __restrict__ st,
                                                           float* __restrict__ hlr /*[2][W][H]*/) {
     extern __shared__ float sm_rnn[];
     float* state = sm_rnn;
@@ -185,18 +201,19 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float* Wh = dir ? m.Whb : m.Whf;
     const float* init = dir ? m.b0 : m.a0;
+    const uint32_t pushes = st->push_count;
+    const float inv_scale = st->inv_scale;
     for (int i = threadIdx.x; i < m.H; i += kRnnThreads) state[i] = init[i];
     __syncthreads();
     for (int s = 0; s < m.W; ++s) {
         const int t = dir ? (m.W - 1 - s) : s;
-        const float* p = proj + (static_cast<size_t>(dir) * m.W + t) * m.H;
         for (int i = warp; i < m.H; i += kRnnThreads / 32) {
             const float* wrow = Wh + static_cast<size_t>(i) * m.H;
             float acc = 0.0f;
             for (int j = lane; j < m.H; j += 32) acc = fmaf(wrow[j], state[j], acc);
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-            if (lane == 0) next[i] = fmaxf(acc + p[i], 0.0f);
+            if (lane == 0) next[i] = fmaxf(acc + window_projection(m, proj, dir, t, i, pushes, inv_scale), 0.0f);
         }
         __syncthreads();
         float* out = hlr + (static_cast<size_t>(dir) * m.W + t) * m.H;
@@ -219,6 +236,7 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
 template <int HQ>   // HQ = H / 4
 __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const float* __restrict__ wh_threads,
                                                               const float* __restrict__ proj,
+                                                              const DevState* __restrict__ dev_state,
                                                               float* __restrict__ hlr /*[2][W][H]*/) {
     constexpr int H = 4 * HQ, T = 16 * HQ, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ, PAD = HQ + 4;
     extern __shared__ __align__(16) float sm_rr[];
@@ -240,7 +258,11 @@ __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const 
 #pragma unroll
     for (int j4 = 0; j4 < SQ / 4; ++j4)
         *reinterpret_cast<float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4) = Wh[static_cast<size_t>(RQ / 4 + j4) * T + t];
-    for (int idx = t; idx < m.W * H; idx += T) sproj[idx] = proj[static_cast<size_t>(dir) * m.W * H + idx];
+    {
+        const uint32_t pushes = dev_state->push_count;
+        const float inv_scale = dev_state->inv_scale;
+        for (int idx = t; idx < m.W * H; idx += T) sproj[idx] = window_projection(m, proj, dir, idx / H, idx % H, pushes, inv_scale);
+    }
     if (t < H) state[(t / HQ) * PAD + (t % HQ)] = init[t];
     __syncthreads();
     int cur = 0;

@@ -475,24 +475,25 @@ __global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restr
 // ---------------------------------------------------------------------------------------------
 // Column sums of the partial rows, in a fixed order, in double, followed by the decision in the
 // CTA that finishes last (a ticket counter in the device state; nobody waits on anybody).
-// A CTA covers 32 columns with 8 row slices; slice s adds rows s, s+8, ...; the slices are then
+// A CTA covers 32 columns with 32 row slices; slice s adds rows s, s+32, ...; the slices are then
 // added in order.
 // ---------------------------------------------------------------------------------------------
-constexpr int kColsumThreads = 256;
+constexpr int kColsumSlices = 32;
+constexpr int kColsumThreads = 32 * kColsumSlices;
 
 __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* __restrict__ partial, int n_part, int N,
                                                                    double* sums, double inv_samples, DevState* st,
                                                                    float* __restrict__ e_out, float* __restrict__ omega_out,
                                                                    const float* __restrict__ partial_sq,
                                                                    float* __restrict__ std_out) {
-    __shared__ double red[8][32];
+    __shared__ double red[kColsumSlices][32];
     __shared__ bool is_last;
     const int col = blockIdx.x * 32 + (threadIdx.x & 31), slice = threadIdx.x >> 5;
     if (partial_sq) {
         // spread of each order statistic over the samples: sqrt(E[x^2] - E[x]^2), in seconds
         double s1 = 0.0, s2 = 0.0;
         if (col < N)
-            for (int p = slice; p < n_part; p += 8) {
+            for (int p = slice; p < n_part; p += kColsumSlices) {
                 s1 += static_cast<double>(partial[static_cast<size_t>(p) * N + col]);
                 s2 += static_cast<double>(partial_sq[static_cast<size_t>(p) * N + col]);
             }
@@ -500,13 +501,13 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
         __syncthreads();
         double t1 = 0.0;
         if (slice == 0)
-            for (int k = 0; k < 8; ++k) t1 += red[k][threadIdx.x];
+            for (int k = 0; k < kColsumSlices; ++k) t1 += red[k][threadIdx.x];
         __syncthreads();
         red[slice][threadIdx.x & 31] = s2;
         __syncthreads();
         if (slice == 0 && col < N) {
             double t2 = 0.0;
-            for (int k = 0; k < 8; ++k) t2 += red[k][threadIdx.x];
+            for (int k = 0; k < kColsumSlices; ++k) t2 += red[k][threadIdx.x];
             const double mean = t1 * inv_samples, var = t2 * inv_samples - mean * mean;
             std_out[col] = static_cast<float>(static_cast<double>(st->scale) * sqrt(var > 0.0 ? var : 0.0));
         }
@@ -515,24 +516,24 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
     double s = 0.0;
     if (col < N) {
         int p = slice;
-        for (; p + 24 < n_part; p += 32) {
+        for (; p + 3 * kColsumSlices < n_part; p += 4 * kColsumSlices) {        // four loads in flight
             const float a = partial[static_cast<size_t>(p) * N + col];
-            const float b = partial[static_cast<size_t>(p + 8) * N + col];
-            const float c = partial[static_cast<size_t>(p + 16) * N + col];
-            const float d = partial[static_cast<size_t>(p + 24) * N + col];
+            const float b = partial[static_cast<size_t>(p + kColsumSlices) * N + col];
+            const float c = partial[static_cast<size_t>(p + 2 * kColsumSlices) * N + col];
+            const float d = partial[static_cast<size_t>(p + 3 * kColsumSlices) * N + col];
             s += static_cast<double>(a);
             s += static_cast<double>(b);
             s += static_cast<double>(c);
             s += static_cast<double>(d);
         }
-        for (; p < n_part; p += 8) s += static_cast<double>(partial[static_cast<size_t>(p) * N + col]);
+        for (; p < n_part; p += kColsumSlices) s += static_cast<double>(partial[static_cast<size_t>(p) * N + col]);
     }
     red[slice][threadIdx.x & 31] = s;
     __syncthreads();
     if (slice == 0 && col < N) {
         double total = 0.0;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) total += red[k][threadIdx.x];
+        for (int k = 0; k < kColsumSlices; ++k) total += red[k][threadIdx.x];
         sums[col] = total;
     }
     __threadfence();
