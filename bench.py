@@ -36,8 +36,10 @@ MINMAX_LANES_PER_SM = 64         # fp32 min / max lanes per SM per clock (ALU pi
 # DRAM bytes per launch of the dominant kernel, from the ncu capture summarised under profiles/ (valid for the
 # kernel as committed with that summary; set to None when the kernel changes).
 NCU_TRAFFIC = {
-    ("n1024", "sort"): {"bytes_per_sample": (201392896 + 4176896) / 49152,
+    ("n1024", "sort"): {"bytes_per_sample": (201393408 + 3632128) / 49152,
                         "source": "profiles/ncu_full_n1024_s49152_chain_emit_sort.txt (S=49152, scaled by S)"},
+    ("n4096", "sort"): {"bytes_per_sample": (134251776 + 8298752) / 8192,
+                        "source": "profiles/ncu_full_n4096_s8192_sort.txt (S=8192, scaled by S)"},
 }
 PRECISION_NAMES = {0: "f32", 1: "tf32", 2: "tf32(bf16 weights)"}
 
