@@ -34,11 +34,12 @@ SM_COUNT = 148
 FP32_LANES_PER_SM = 128          # fused multiply-add lanes per SM per clock
 MINMAX_LANES_PER_SM = 64         # fp32 min / max lanes per SM per clock (ALU pipe: 16 per sub-partition)
 # DRAM bytes per launch of the dominant kernel, from the ncu capture summarised under profiles/ (valid for the
-# kernel as committed with that summary; set to None when the kernel changes).
+# kernel as committed with that summary; set to None when the kernel changes): the sample matrix read once
+# (grows with S) plus the partial rows written (one per CTA: does not grow with S).
 NCU_TRAFFIC = {
-    ("n1024", "sort"): {"bytes_per_sample": (201393408 + 3632128) / 49152,
+    ("n1024", "sort"): {"bytes_per_sample": 201393408 / 49152, "bytes_fixed": 3632128,
                         "source": "profiles/ncu_full_n1024_s49152_chain_emit_sort.txt (S=49152, scaled by S)"},
-    ("n4096", "sort"): {"bytes_per_sample": (134251776 + 8298752) / 8192,
+    ("n4096", "sort"): {"bytes_per_sample": 134251776 / 8192, "bytes_fixed": 8298752,
                         "source": "profiles/ncu_full_n4096_s8192_sort.txt (S=8192, scaled by S)"},
 }
 PRECISION_NAMES = {0: "f32", 1: "tf32", 2: "tf32(bf16 weights)"}
@@ -362,7 +363,7 @@ def main():
     achieved = amount / dur / 1e12
     traffic = None if literal else NCU_TRAFFIC.get((wl.name, dominant))
     roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
-                "frac": achieved / peak, "traffic": traffic["bytes_per_sample"] * wl.S if traffic else None,
+                "frac": achieved / peak, "traffic": traffic["bytes_per_sample"] * wl.S + traffic["bytes_fixed"] if traffic else None,
                 "traffic_source": traffic["source"] if traffic else None,
                 "algorithmic_per_launch": amount, "peak_source": peak_src,
                 "stage_ms": {k: round(v, 4) for k, v in stage_avg.items()}}
