@@ -467,3 +467,29 @@ def test_degenerate_and_equal_times():
     e, om = gpu.get_stats()
     s = 2.0 * inputs.workload_trace(wl, 3)[:2].astype(np.float64).mean()
     assert np.allclose(e, 0.75 * s, rtol=1e-6)
+
+
+@pytest.mark.parametrize("N,D,H,lag,S,prec", [(32, 4, 1024, 1, 200, 0), (8, 4, 32, 255, 64, 0), (4096, 4, 16, 0, 40, 0),
+                                               (96, 32, 512, 3, 150, 1), (64, 8, 1024, 0, 130, 2)])
+def test_limits_of_the_supported_shapes(N, D, H, lag, S, prec):
+    # the widest hidden layer, the longest window, the most workers, the widest tensor-core chain
+    w = inputs.make_weights(N, D, H, seed=5, fan_in_ref=32, bf16=(prec == 2))
+    trace = inputs.make_trace(N, lag + 3, seed=11, sigma=0.2)
+    gpu = binding.Cutoff(N, D, H, lag, S, precision=prec, seed=SEED)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, lag, S, seed=SEED)
+    for x in trace:
+        gpu.push(x)
+        orc.push(x)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec] if prec else 2e-5)
+    assert_decision_close(gpu, orc.predict(), N)
+
+
+@pytest.mark.parametrize("kw", [dict(n_workers=4097), dict(latent_dim=5), dict(latent_dim=64), dict(hidden=1028),
+                                dict(hidden=30), dict(lag=256), dict(latent_dim=32, hidden=1024)])
+def test_unsupported_shapes_are_refused(kw):
+    args = dict(n_workers=64, latent_dim=8, hidden=64, lag=1, n_samples=64)
+    args.update(kw)
+    with pytest.raises(binding.CutoffError) as e:
+        binding.Cutoff(**args)
+    assert e.value.code in (binding.ERR_UNSUPPORTED, binding.ERR_BAD_ARG)
