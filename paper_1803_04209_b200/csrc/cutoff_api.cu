@@ -453,8 +453,20 @@ void launch_encoder(cutoff_ctx* c) {
         case 64: launch_rnn_resident<16>(c); break;
         case 128: launch_rnn_resident<32>(c); break;
         case 256: launch_rnn_resident<64>(c); break;
-        default:
-            k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
+        default: {
+            const size_t cluster_smem = enc_rnn_cluster_smem_floats(c->H, c->W) * sizeof(float);
+            if (!fits && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024) {
+                // the matrix of a direction split over a cluster of 8 CTAs
+                static bool attr_set = false;
+                if (!attr_set) {
+                    cudaFuncSetAttribute(k_enc_rnn_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+                    attr_set = true;
+                }
+                k_enc_rnn_cluster<<<2 * kRnnClusterSize, c->H, cluster_smem, c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
+            } else {
+                k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
+            }
+        }
     }
     c->launches += 1;
 }

@@ -301,6 +301,80 @@ inline size_t enc_rnn_resident_smem_floats(int H, int W) {
 }
 
 // ---------------------------------------------------------------------------------------------
+// Encoder, part 2, for 256 < H <= 640: the recurrence matrix of a direction is split over the shared
+// memories of a cluster of 8 CTAs (H/8 rows each), so it is read from global memory once.  Every CTA
+// keeps the whole state (double-buffered); after a step each row's new value is written into the next
+// state buffer of all 8 CTAs through distributed shared memory, and one cluster barrier (a hardware
+// barrier: no thread leaves before the last step) separates the steps.
+// 8 threads per row: thread p of a row takes the 16-byte column chunks p, p+8, ...; rows are padded by
+// 8 floats so that the four rows of a warp fall into different banks.  Grid: 16 CTAs (2 clusters).
+// ---------------------------------------------------------------------------------------------
+constexpr int kRnnClusterSize = 8;
+
+inline size_t enc_rnn_cluster_smem_floats(int H, int W) {
+    const int R = H / kRnnClusterSize;
+    return static_cast<size_t>(R) * (H + 8) + 2 * static_cast<size_t>(H) + static_cast<size_t>(W) * R;
+}
+
+__global__ void __cluster_dims__(kRnnClusterSize, 1, 1) __launch_bounds__(1024)
+k_enc_rnn_cluster(ModelDev m, const float* __restrict__ proj, const DevState* __restrict__ dev_state,
+                  float* __restrict__ hlr /*[2][W][H]*/) {
+    extern __shared__ __align__(16) float sm_rc[];
+    const int H = m.H, W = m.W, R = H / kRnnClusterSize, ldw = H + 8;
+    float* sW = sm_rc;                         // [R][ldw]  rows rank*R .. of the recurrence matrix
+    float* state = sW + static_cast<size_t>(R) * ldw;      // [2][H]
+    float* sproj = state + 2 * H;              // [W][R]
+    uint32_t rank;
+    asm("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int dir = blockIdx.x / kRnnClusterSize;
+    const int row = threadIdx.x >> 3, part = threadIdx.x & 7;          // blockDim.x = 8 R
+    const int i = static_cast<int>(rank) * R + row;                    // hidden unit of this thread's row
+    const float* Wh = (dir ? m.Whb : m.Whf) + static_cast<size_t>(rank) * R * H;
+    const float* init = dir ? m.b0 : m.a0;
+    for (int idx = threadIdx.x; idx < R * (H / 4); idx += blockDim.x) {
+        const int r = idx / (H / 4), c = idx % (H / 4);
+        *reinterpret_cast<float4*>(sW + static_cast<size_t>(r) * ldw + 4 * c) =
+            *reinterpret_cast<const float4*>(Wh + static_cast<size_t>(r) * H + 4 * c);
+    }
+    for (int k = threadIdx.x; k < H; k += blockDim.x) state[k] = init[k];
+    {
+        const uint32_t pushes = dev_state->push_count;
+        const float inv_scale = dev_state->inv_scale;
+        for (int idx = threadIdx.x; idx < W * R; idx += blockDim.x)
+            sproj[idx] = window_projection(m, proj, dir, idx / R, static_cast<int>(rank) * R + idx % R, pushes, inv_scale);
+    }
+    // every CTA of the cluster has started and initialised its buffers before anyone writes into them
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    const float* wrow = sW + static_cast<size_t>(row) * ldw;
+    int cur = 0;
+    for (int s = 0; s < W; ++s) {
+        const int t = dir ? (W - 1 - s) : s;
+        const float* st = state + cur * H;
+        float acc = 0.0f;
+        for (int c = part; c < H / 4; c += 8) {
+            const float4 w = *reinterpret_cast<const float4*>(wrow + 4 * c);
+            const float4 v = *reinterpret_cast<const float4*>(st + 4 * c);
+            acc = fmaf(w.x, v.x, acc); acc = fmaf(w.y, v.y, acc);
+            acc = fmaf(w.z, v.z, acc); acc = fmaf(w.w, v.w, acc);
+        }
+        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+        acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+        const float v = fmaxf(acc + sproj[t * R + row], 0.0f);
+        // thread `part` of the row delivers the new value to CTA `part` of the cluster
+        {
+            const uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(state + (cur ^ 1) * H + i));
+            uint32_t remote;
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(static_cast<uint32_t>(part)));
+            asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(remote), "f"(v) : "memory");
+        }
+        if (part == 0) hlr[(static_cast<size_t>(dir) * W + t) * H + i] = v;
+        asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+        cur ^= 1;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Per-sample chain: guide steps over the window, transition, first emission layer.
 //
 // SPL samples are worked on by a group of G = D/4 adjacent lanes.  Lane g of the group owns, of
