@@ -16,6 +16,7 @@
 #include "chain_tc32.cuh"
 #include "kernels_literal.cuh"
 #include "gemm_tc.cuh"
+#include "chain_tc_literal.cuh"
 
 using namespace cutoff;
 
@@ -82,6 +83,7 @@ struct cutoff_ctx {
     bool use_tc = false;            // emission output layer on tensor cores
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
     bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
+    bool chain_tcl = false;         // the literal variant's chain on tensor cores (D = 16, H in {64, 128, 192, 256})
     float* d_chain_image = nullptr; // swizzled tf32 operand tiles of the chain
 
     float* h_stage = nullptr;       // pinned [N]
@@ -300,7 +302,29 @@ void launch_chain_literal_t(cutoff_ctx* c, uint32_t sample_base, int count) {
         c->m, c->lit, c->d_hlr, c->d_state, key, sample_base, count, c->use_tc ? 1 : 0, c->d_v);
 }
 
+void launch_chain_tc_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaFuncSetAttribute(tc::k_chain_tc_literal, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        attr_set = true;
+    }
+    tc::ChainTclArgs a;
+    const ModelDev& m = c->m;
+    const LiteralDev& l = c->lit;
+    a.image = c->d_chain_image;
+    a.bz = m.bz; a.bg1 = l.bg1; a.bh1 = l.bh1; a.bi1 = l.bi1; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig;
+    a.bg2 = l.bg2; a.bh2 = l.bh2; a.Wl = l.Wl; a.bl = l.bl; a.bs = l.bs; a.z0 = m.z0;
+    a.hlr = c->d_hlr; a.st = c->d_state;
+    a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
+    a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.u_out = c->d_v;
+    const int tiles = ceil_div(count, 128);
+    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
+    tc::k_chain_tc_literal<<<grid, tc::kChainTcThreads, tc::chain_tcl_smem_bytes(c->H, c->W), c->stream>>>(a);
+    c->launches += 1;
+}
+
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
+    if (c->chain_tcl) { launch_chain_tc_literal(c, sample_base, count); return; }
     if (c->literal) {
         switch (c->D) {
             case 4: launch_chain_literal_t<4>(c, sample_base, count); break;
@@ -611,6 +635,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     c->use_tc = cfg->precision != CUTOFF_PRECISION_FP32;
     c->chain_tc = !c->literal && c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
                   tc::chain_tc_smem_bytes(c->H, c->W) <= 227 * 1024;
+    c->chain_tcl = c->literal && c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
+                   tc::chain_tcl_smem_bytes(c->H, c->W) <= 227 * 1024;
     c->chain_tc32 = !c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
                     (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W) <= 227 * 1024;
 
@@ -629,6 +655,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     if (c->chain_tc32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H)));
+    if (c->chain_tcl) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tcl_image_floats(c->H)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_mask, c->N));
@@ -779,6 +806,47 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
                 for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
                 for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + at(o, jj)] = tf32(w2[o * H + kb * 32 + jj]);
             }
+        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+
+    if (c->chain_tcl) {
+        // Literal variant, D = 16: [Wz | Wg1] and [Wh1 | Wi1] as [H rows][32], Wmu, Wg2, Wh2 as H/32 K blocks of
+        // [16 rows][32], Ws as [16 rows][32] (columns 16.. zero), all tf32 in the swizzled shared-memory layout.
+        auto tf32 = [](float f) {
+            uint32_t u;
+            std::memcpy(&u, &f, 4);
+            u = (u + 0x1000u) & 0xFFFFE000u;
+            std::memcpy(&f, &u, 4);
+            return f;
+        };
+        auto at = [](size_t row, size_t col) {
+            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
+        };
+        std::vector<float> img(tc::chain_tcl_image_floats(c->H), 0.0f);
+        const float* wz = host.data() + off[8];      // [H][D]
+        const float* wg1 = host.data() + off[15];
+        const float* wh1 = host.data() + off[19];
+        const float* wi1 = host.data() + off[27];
+        const float* second[3] = {host.data() + off[10], host.data() + off[17], host.data() + off[21]};   // Wmu, Wg2, Wh2: [D][H]
+        const float* ws = host.data() + off[25];     // [D][D]
+        float* t_zg = img.data();
+        float* t_hi = t_zg + H * 32;
+        float* t_second = t_hi + H * 32;             // three tiles of H x 16 floats
+        float* t_ws = t_second + 3 * H * 16;
+        for (size_t n = 0; n < H; ++n)
+            for (size_t k = 0; k < D; ++k) {
+                t_zg[at(n, k)] = tf32(wz[n * D + k]);
+                t_zg[at(n, 16 + k)] = tf32(wg1[n * D + k]);
+                t_hi[at(n, k)] = tf32(wh1[n * D + k]);
+                t_hi[at(n, 16 + k)] = tf32(wi1[n * D + k]);
+            }
+        for (int t = 0; t < 3; ++t)
+            for (size_t kb = 0; kb < H / 32; ++kb)
+                for (size_t jj = 0; jj < 32; ++jj)
+                    for (size_t d = 0; d < D; ++d)
+                        t_second[t * H * 16 + kb * 16 * 32 + at(d, jj)] = tf32(second[t][d * H + kb * 32 + jj]);
+        for (size_t o = 0; o < D; ++o)
+            for (size_t e = 0; e < D; ++e) t_ws[at(o, e)] = tf32(ws[o * D + e]);
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
 
