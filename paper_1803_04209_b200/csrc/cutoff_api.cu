@@ -418,8 +418,25 @@ void launch_emission_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
         launch_gemm_tc<kEpiAffine>(c, c->map_v, c->map_wi2, a);
         a.bias = l.bj1; a.out = c->d_r; a.ld_out = c->H; a.Nout = c->H; a.K = c->N; a.round_out = 1;
         launch_gemm_tc<kEpiRelu>(c, c->map_I, c->map_wj1, a);
-        a.bias = l.bj2; a.add = c->d_I; a.out = c->d_x; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H; a.round_out = 0;
-        launch_gemm_tc<kEpiScaleNoise>(c, c->map_r, c->map_wj2, a);
+        if (c->H > 256) {
+            // wide hidden layers: the products are bound by the tensor pipe, so I is read back rather than recomputed
+            a.bias = l.bj2; a.add = c->d_I; a.out = c->d_x; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H; a.round_out = 0;
+            launch_gemm_tc<kEpiScaleNoise>(c, c->map_r, c->map_wj2, a);
+            return;
+        }
+        // third product fused with a recomputation of I in the same accumulator (I is not read back)
+        static bool attr_set = false;
+        if (!attr_set) {
+            cudaFuncSetAttribute(tc::k_emit_dual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kDualSmemBytes));
+            attr_set = true;
+        }
+        tc::EmitDualArgs e;
+        e.bias_mean = l.bi2; e.bias_scale = l.bj2; e.x = c->d_x; e.st = c->d_state; e.key = key;
+        e.sample_base = sample_base; e.count = count; e.N = c->N; e.H = c->H; e.ldx = c->ldx;
+        const int tiles = ceil_div(c->N, tc::kBW) * ceil_div(count, tc::kBM);
+        tc::k_emit_dual_tc<<<tiles < c->sm_count ? tiles : c->sm_count, tc::kThreads, tc::kDualSmemBytes, c->stream>>>(
+            c->map_v, c->map_r, c->map_wi2, c->map_wj2, e);
+        c->launches += 1;
         return;
     }
     GemmFmaArgs a{};
