@@ -74,9 +74,11 @@ def stage_work(wl, S, literal=False):
         p *= 2
     chain = S * (W * (2 * D * H + D * D) + 3 * D * H + D * H)
     emit_macs = S * H * 2 * N
-    if literal:      # gate and proposal (2 x 2DH), linear map and scale (2 x D^2), first emission layer; three N x H products
+    if literal:      # gate and proposal (2 x 2DH), linear map and scale (2 x D^2), first emission layer
         chain = S * (W * (2 * D * H + D * D) + 4 * D * H + 2 * D * D + D * H)
-        emit_macs = S * H * 3 * N
+        # fp32: three N x H products; tensor cores: the scale's hidden layer as one H x H product (I is affine in u),
+        # then the mean and the scale product in one accumulator
+        emit_macs = S * H * (2 * N + H) if wl.precision else S * H * 3 * N
     return {
         "encoder": ("alu", 2 * W * (N * H + H * H)),
         "chain": ("alu", chain),

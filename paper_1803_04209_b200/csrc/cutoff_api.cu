@@ -75,11 +75,12 @@ struct cutoff_ctx {
 
     bool literal = false;           // the networks as Section 3.1.3 prints them (CUTOFF_FLAG_LITERAL)
     LiteralDev lit{};
-    float* d_I = nullptr;           // [alloc_rows][ldx]  emission mean I (padding columns stay zero)
+    float* d_I = nullptr;           // [alloc_rows][ldx]  emission mean I (padding columns stay zero); fp32 path only
     float* d_r = nullptr;           // [alloc_rows][H]    hidden layer of the emission scale
-    float* d_Wj1p = nullptr;        // [H][ldx]           Wj1 with rows padded with zeros to ldx
-    CUtensorMap map_I{}, map_r{};   // TMA views of d_I [alloc_rows][N] and d_r [alloc_rows][H]
-    CUtensorMap map_wi2{}, map_wj1{}, map_wj2{};
+    float* d_Wj1p = nullptr;        // [H][ldx]           Wj1 with rows padded with zeros to ldx; fp32 path only
+    float* d_M = nullptr;           // [H][H] then [H]    M = Wj1 Wi2 and b' = Wj1 bi2 + bj1 (tensor-core path: Wj1 I + bj1 = M u + b')
+    CUtensorMap map_r{};            // TMA view of d_r [alloc_rows][H]
+    CUtensorMap map_wi2{}, map_M{}, map_wj2{};
     bool use_tc = false;            // emission output layer on tensor cores
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
     bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
@@ -153,7 +154,7 @@ int next_pow2(int n) {
 }
 
 void free_all(cutoff_ctx* c) {
-    cudaFree(c->d_I); cudaFree(c->d_r); cudaFree(c->d_Wj1p);
+    cudaFree(c->d_I); cudaFree(c->d_r); cudaFree(c->d_Wj1p); cudaFree(c->d_M);
     cudaFree(c->d_blob); cudaFree(c->d_WT); cudaFree(c->d_WhR); cudaFree(c->d_chain_image); cudaFree(c->d_mask);
     if (c->h_mask) cudaFreeHost(c->h_mask); cudaFree(c->d_ring); cudaFree(c->d_stage);
     cudaFree(c->d_state); cudaFree(c->d_proj); cudaFree(c->d_hlr); cudaFree(c->d_v); cudaFree(c->d_x);
@@ -395,16 +396,15 @@ void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
 }
 
 // Literal emission (Section 3.1.3): I = u Wi2^T + bi2, r = relu(I Wj1^T + bj1), x = I + softplus(r Wj2^T + bj2) * eps.
-template <int EPI>
-void launch_gemm_tc(cutoff_ctx* c, const CUtensorMap& map_a, const CUtensorMap& map_b, const tc::GemmTcArgs& a) {
+void launch_gemm_relu_tc(cutoff_ctx* c, const CUtensorMap& map_a, const CUtensorMap& map_b, const tc::GemmTcArgs& a) {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_gemm_tc<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
+        cudaFuncSetAttribute(tc::k_gemm_relu_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
         attr_set = true;
     }
     const int tiles = ceil_div(a.Nout, tc::kGemmBN) * ceil_div(a.M, tc::kBM);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    tc::k_gemm_tc<EPI><<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(map_a, map_b, a);
+    tc::k_gemm_relu_tc<<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(map_a, map_b, a);
     c->launches += 1;
 }
 
@@ -412,19 +412,11 @@ void launch_emission_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     const LiteralDev& l = c->lit;
     if (c->use_tc) {
+        // r = relu(M u + b') with M = Wj1 Wi2 (I is affine in u), then x = (Wi2 u + bi2) + softplus(Wj2 r + bj2) * eps
         tc::GemmTcArgs a{};
-        a.st = c->d_state; a.key = key; a.sample_base = sample_base; a.M = count;
-        a.bias = l.bi2; a.out = c->d_I; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H;
-        launch_gemm_tc<kEpiAffine>(c, c->map_v, c->map_wi2, a);
-        a.bias = l.bj1; a.out = c->d_r; a.ld_out = c->H; a.Nout = c->H; a.K = c->N; a.round_out = 1;
-        launch_gemm_tc<kEpiRelu>(c, c->map_I, c->map_wj1, a);
-        if (c->H > 256) {
-            // wide hidden layers: the products are bound by the tensor pipe, so I is read back rather than recomputed
-            a.bias = l.bj2; a.add = c->d_I; a.out = c->d_x; a.ld_out = c->ldx; a.Nout = c->N; a.K = c->H; a.round_out = 0;
-            launch_gemm_tc<kEpiScaleNoise>(c, c->map_r, c->map_wj2, a);
-            return;
-        }
-        // third product fused with a recomputation of I in the same accumulator (I is not read back)
+        a.st = c->d_state; a.M = count; a.bias = c->d_M + static_cast<size_t>(c->H) * c->H; a.out = c->d_r;
+        a.ld_out = c->H; a.Nout = c->H; a.K = c->H;
+        launch_gemm_relu_tc(c, c->map_v, c->map_M, a);
         static bool attr_set = false;
         if (!attr_set) {
             cudaFuncSetAttribute(tc::k_emit_dual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kDualSmemBytes));
@@ -643,7 +635,10 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
 
     // Pass buffers hold up to 2 GiB of samples; by default one pass covers all S samples.
     {
-        int64_t cap = (2ll << 30) / (static_cast<int64_t>(c->ldx + c->H) * (c->literal ? 2 : 1) * sizeof(float));
+        // per sample: x and v; literal variant: also r, and I on the fp32 path
+        const bool tensor_path = cfg->precision != CUTOFF_PRECISION_FP32;
+        const int64_t row_floats = c->ldx + c->H + (c->literal ? c->H + (tensor_path ? 0 : c->ldx) : 0);
+        int64_t cap = (2ll << 30) / (row_floats * static_cast<int64_t>(sizeof(float)));
         if (cap < 1024) cap = 1024;
         c->alloc_rows = cap < c->S ? static_cast<int>(cap) : c->S;
     }
@@ -663,11 +658,15 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_blob, blob_floats * sizeof(float)));
     CREATE_CHECK(cudaMalloc(&c->d_WT, sizeof(float) * 4 * c->H * c->D));
     if (c->literal) {
-        CREATE_CHECK(cudaMalloc(&c->d_I, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
         CREATE_CHECK(cudaMalloc(&c->d_r, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->H));
-        CREATE_CHECK(cudaMalloc(&c->d_Wj1p, sizeof(float) * static_cast<size_t>(c->H) * c->ldx));
-        // the padding columns of I are never written and must read as zero
-        CREATE_CHECK(cudaMemsetAsync(c->d_I, 0, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx, c->stream));
+        if (c->use_tc) {
+            CREATE_CHECK(cudaMalloc(&c->d_M, sizeof(float) * (static_cast<size_t>(c->H) * c->H + c->H)));
+        } else {
+            CREATE_CHECK(cudaMalloc(&c->d_I, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx));
+            CREATE_CHECK(cudaMalloc(&c->d_Wj1p, sizeof(float) * static_cast<size_t>(c->H) * c->ldx));
+            // the padding columns of I are never written and must read as zero
+            CREATE_CHECK(cudaMemsetAsync(c->d_I, 0, sizeof(float) * static_cast<size_t>(c->alloc_rows) * c->ldx, c->stream));
+        }
     }
     CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
@@ -690,8 +689,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     if (c->use_tc) {
         int rc = make_tile_map(c, &c->map_v, c->d_v, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
         if (!rc && c->literal)
-            rc = make_tile_map(c, &c->map_I, c->d_I, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->N),
-                               static_cast<uint64_t>(c->ldx));
+            rc = make_tile_map(c, &c->map_M, c->d_M, static_cast<uint64_t>(c->H), static_cast<uint64_t>(c->H));
         if (!rc && c->literal)
             rc = make_tile_map(c, &c->map_r, c->d_r, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
         if (rc) return fail(rc);
@@ -911,11 +909,43 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     m.WzT = c->d_WT; m.bz = b + off[9]; m.Wmu = b + off[10]; m.bmu = b + off[11];
     m.Wsig = b + off[12]; m.bsig = b + off[13]; m.z0 = b + off[14];
     if (c->literal) {
-        // Wj1 [H][N] with rows padded with zeros to ldx floats (rows then start on 32 bytes for any N)
-        std::vector<float> wj1p(H * static_cast<size_t>(c->ldx), 0.0f);
-        for (size_t i = 0; i < H; ++i)
-            std::memcpy(wj1p.data() + i * c->ldx, host.data() + off[31] + i * c->N, sizeof(float) * c->N);
-        CU_CHECK(c, cudaMemcpy(c->d_Wj1p, wj1p.data(), wj1p.size() * sizeof(float), cudaMemcpyHostToDevice));
+        if (c->use_tc) {
+            // I = Wi2 u + bi2 is affine in u, so Wj1 I + bj1 = M u + b' with M = Wj1 Wi2 [H][H] and b' = Wj1 bi2 + bj1:
+            // formed here once, in double, from the weights as the tensor cores see them; M is rounded to tf32.
+            const size_t N = c->N;
+            const float* wj1 = host.data() + off[31];    // [H][N]
+            const float* wi2 = host.data() + off[29];    // [N][H]
+            const float* bi2 = host.data() + off[30];
+            const float* bj1 = host.data() + off[32];
+            std::vector<float> mb(H * H + H);
+            std::vector<double> acc(H);
+            for (size_t i = 0; i < H; ++i) {
+                std::fill(acc.begin(), acc.end(), 0.0);
+                double bacc = bj1[i];
+                for (size_t k = 0; k < N; ++k) {
+                    const double w = wj1[i * N + k];
+                    const float* row = wi2 + k * H;
+                    for (size_t j = 0; j < H; ++j) acc[j] += w * row[j];
+                    bacc += w * bi2[k];
+                }
+                for (size_t j = 0; j < H; ++j) {
+                    float f = static_cast<float>(acc[j]);
+                    uint32_t u;
+                    std::memcpy(&u, &f, 4);
+                    u = (u + 0x1000u) & 0xFFFFE000u;
+                    std::memcpy(&f, &u, 4);
+                    mb[i * H + j] = f;
+                }
+                mb[H * H + i] = static_cast<float>(bacc);
+            }
+            CU_CHECK(c, cudaMemcpy(c->d_M, mb.data(), mb.size() * sizeof(float), cudaMemcpyHostToDevice));
+        } else {
+            // Wj1 [H][N] with rows padded with zeros to ldx floats (rows then start on 32 bytes for any N)
+            std::vector<float> wj1p(H * static_cast<size_t>(c->ldx), 0.0f);
+            for (size_t i = 0; i < H; ++i)
+                std::memcpy(wj1p.data() + i * c->ldx, host.data() + off[31] + i * c->N, sizeof(float) * c->N);
+            CU_CHECK(c, cudaMemcpy(c->d_Wj1p, wj1p.data(), wj1p.size() * sizeof(float), cudaMemcpyHostToDevice));
+        }
         LiteralDev& l = c->lit;
         l.Wg1T = c->d_WT + H * D; l.bg1 = b + off[16]; l.Wg2 = b + off[17]; l.bg2 = b + off[18];
         l.Wh1T = c->d_WT + 2 * H * D; l.bh1 = b + off[20]; l.Wh2 = b + off[21]; l.bh2 = b + off[22];
@@ -927,8 +957,6 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         m.W1T = m.b1 = m.W2 = m.b2 = m.W3T = m.b3 = m.W4 = m.b4 = nullptr;
         if (c->use_tc) {
             int rc = make_tile_map(c, &c->map_wi2, l.Wi2, static_cast<uint64_t>(c->N), static_cast<uint64_t>(c->H));
-            if (!rc) rc = make_tile_map(c, &c->map_wj1, l.Wj1, static_cast<uint64_t>(c->H), static_cast<uint64_t>(c->N),
-                                        static_cast<uint64_t>(c->ldx));
             if (!rc) rc = make_tile_map(c, &c->map_wj2, l.Wj2, static_cast<uint64_t>(c->N), static_cast<uint64_t>(c->H));
             if (rc) return rc;
         }

@@ -1,8 +1,12 @@
-// C = A B^T with an epilogue on the 5th-generation tensor cores (tcgen05, kind::tf32): the three
-// matrix products of the literal emission of Section 3.1.3,
-//   I = u Wi2^T + bi2        r = relu(I Wj1^T + bj1)        x = I + softplus(r Wj2^T + bj2) * eps.
+// The emission of the literal model variant (Section 3.1.3) on the 5th-generation tensor cores (tcgen05, kind::tf32):
+//   I = Wi2 u + bi2        r = relu(Wj1 I + bj1)        x = I + softplus(Wj2 r + bj2) * eps,      u = Wi1 z' + bi1.
+// I = MLP_2(z, Identity, Identity) is affine in u, so the hidden layer of the scale does not need I:
+//   Wj1 I + bj1 = (Wj1 Wi2) u + (Wj1 bi2 + bj1) = M u + b',
+// with the H x H matrix M and the vector b' formed once when the weights are loaded.  Two kernels remain:
+//   k_gemm_relu_tc   r = relu(u M^T + b')                       (K = H instead of K = N)
+//   k_emit_dual_tc   x = (u Wi2^T + bi2) + softplus(r Wj2^T + bj2) * eps,  both products in one accumulator.
 //
-// Same pipeline as the emission kernel of emit_tc.cuh: one persistent CTA per SM walks over output
+// k_gemm_relu_tc has the pipeline of the emission kernel of emit_tc.cuh: one persistent CTA per SM walks over output
 // tiles of 128 rows x 256 columns; a tile is one accumulator of 128 TMEM lanes x 256 fp32 columns,
 // filled by UMMA instructions of shape M=128, N=256, K=8; operands arrive by plain per-CTA TMA loads
 // (boxes of 128 rows x 32 tf32, 128-byte swizzle; rows or columns outside the matrices read as zero)
@@ -22,23 +26,16 @@ constexpr int kGemmBN = 256;              // output columns per tile
 
 struct GemmTcArgs {
     const float* bias;      // [Nout]
-    const float* add;       // [M][ld_out], kEpiScaleNoise only
-    float* out;             // [M][ld_out]
+    float* out;             // [M][ld_out]: relu(A B^T + bias), rounded to tf32 (it is the next product's operand)
     DevState* st;
-    NoiseKey key;
-    uint32_t sample_base;
     int M, Nout, K, ld_out;
-    int round_out;          // kEpiRelu: round the result to tf32 (it is the next product's operand)
 };
 
-template <int EPI>
 __device__ __forceinline__ void gemm_epilogue_tile(const GemmTcArgs& a, uint32_t tmem_base, uint32_t acc, int q, int cg,
-                                                   int lane, int m0, int w0, uint32_t step, uint32_t bar_acc_empty,
-                                                   const float* bias_s) {
+                                                   int lane, int m0, int w0, uint32_t bar_acc_empty, const float* bias_s) {
     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * kAccCols + cg * 32;
     const int row = m0 + q * 32 + lane;
     const bool row_ok = row < a.M;
-    const uint32_t sample = a.sample_base + static_cast<uint32_t>(row);
     const bool wide_store = (a.ld_out & 7) == 0;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
@@ -59,27 +56,11 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmTcArgs& a, uint32_t
             float out[16];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const int j = jw + 4 * i;
-                if (j >= a.Nout) continue;
                 const float4 bv = *reinterpret_cast<const float4*>(bias_s + 32 * part + 16 * half + 4 * i);
                 const float b[4] = {bv.x, bv.y, bv.z, bv.w};
-                float eps[4] = {0.f, 0.f, 0.f, 0.f}, base[4] = {0.f, 0.f, 0.f, 0.f};
-                if (EPI == kEpiScaleNoise) {
-                    normal4_fast(static_cast<uint32_t>(j >> 2), sample, kStreamEmission, step, a.key.seed_lo,
-                                 a.key.seed_hi, eps);
-                    const float4 iv = *reinterpret_cast<const float4*>(a.add + static_cast<size_t>(row) * a.ld_out + j);
-                    base[0] = iv.x; base[1] = iv.y; base[2] = iv.z; base[3] = iv.w;
-                }
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    float v = __uint_as_float(bits[part][4 * i + c]) + b[c];
-                    if (EPI == kEpiRelu) {
-                        v = fmaxf(v, 0.0f);
-                        if (a.round_out) v = round_tf32(v);
-                    }
-                    if (EPI == kEpiScaleNoise) v = fmaf(softplus_fast(v), eps[c], base[c]);
-                    out[4 * i + c] = v;
-                }
+                for (int c = 0; c < 4; ++c)
+                    out[4 * i + c] = round_tf32(fmaxf(__uint_as_float(bits[part][4 * i + c]) + b[c], 0.0f));
             }
 #pragma unroll
             for (int p = 0; p < 2; ++p) {
@@ -102,8 +83,7 @@ __device__ __forceinline__ void gemm_epilogue_tile(const GemmTcArgs& a, uint32_t
     }
 }
 
-template <int EPI>
-__global__ void __launch_bounds__(kThreads, 1) k_gemm_tc(const __grid_constant__ CUtensorMap map_a,
+__global__ void __launch_bounds__(kThreads, 1) k_gemm_relu_tc(const __grid_constant__ CUtensorMap map_a,
                                                           const __grid_constant__ CUtensorMap map_b, GemmTcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -219,7 +199,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_gemm_tc(const __grid_constant__
     } else {
         // ---------------- epilogue ---------------------------------------------------------------
         const int q = warp & 3, cg = (warp - 2) >> 2;
-        const uint32_t step = EPI == kEpiScaleNoise ? a.st->step : 0u;
         float* bias_s = bias_all + (warp - 2) * 64;
         int w_staged = -1;
         uint32_t acc = 0, acc_phase = 0;
@@ -239,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gemm_tc(const __grid_constant__
             ok = mbar_wait(bar_acc_full + 8 * acc, acc_phase, abort_flag, a.st);
             if (!ok) break;
             tc_fence_after();
-            gemm_epilogue_tile<EPI>(a, tmem_base, acc, q, cg, lane, m0, w0, step, bar_acc_empty, bias_s);
+            gemm_epilogue_tile(a, tmem_base, acc, q, cg, lane, m0, w0, bar_acc_empty, bias_s);
             if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
     }
@@ -252,11 +231,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_gemm_tc(const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------------------------
-// The third product fused with a recomputation of the first (used for H <= 256, where the products are not bound
-// by the tensor pipe):  x = I + softplus(r Wj2^T + bj2) * eps  with
-// I = u Wi2^T + bi2 formed again in the same accumulator instead of being read back from memory (reading I
-// back element by element in the epilogue of k_gemm_tc<kEpiScaleNoise> cost 0.14 ms at N=1024, S=65536; the
-// extra multiply-adds run on a tensor pipe that is mostly idle).  Tiles of 128 samples x 128 workers; the
+// x = I + softplus(r Wj2^T + bj2) * eps  with  I = u Wi2^T + bi2, both products in one accumulator, so that I
+// never goes through memory (an earlier version wrote I out and read it back element by element in the epilogue of
+// the scale product: that alone cost 0.14 ms at N=1024, S=65536).  Tiles of 128 samples x 128 workers; the
 // accumulator holds I in columns 0..127 and the scale pre-activation in columns 128..255, from two MMAs per
 // K step with different operands: (u, Wi2 rows) and (r, Wj2 rows).  A stage of the 3-stage ring is
 // [u tile | r tile | Wi2 tile | Wj2 tile], 16 KB each.  Warp roles, accumulator double-buffering and the bounded
