@@ -773,8 +773,9 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     }
     CU_CHECK(c, cudaMemcpy(c->d_WT, wT.data(), wT.size() * sizeof(float), cudaMemcpyHostToDevice));
 
-    {
-        // recurrence matrices regrouped per thread of k_enc_rnn_resident: [dir][j4][thread = 4*i + q][4]
+    if (H == 32 || H == 64 || H == 128 || H == 256) {
+        // recurrence matrices regrouped per thread of k_enc_rnn_resident (the widths that kernel serves; the layout
+        // needs H / 4 to be a multiple of 4): [dir][j4][thread = 4*i + q][4]
         const size_t HQ = H / 4, T = 4 * H;
         std::vector<float> whr(2 * H * H);
         const size_t src_off[2] = {off[1], off[5]};                   // Whf, Whb: each [H][H]

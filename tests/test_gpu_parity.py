@@ -493,3 +493,36 @@ def test_unsupported_shapes_are_refused(kw):
     with pytest.raises(binding.CutoffError) as e:
         binding.Cutoff(**args)
     assert e.value.code in (binding.ERR_UNSUPPORTED, binding.ERR_BAD_ARG)
+
+
+def _random_shapes(n, seed):
+    rng = np.random.default_rng(seed)
+    shapes = []
+    for _ in range(n):
+        D = int(rng.choice([4, 8, 16, 32]))
+        H = D * int(rng.integers(1, 256 // D + 1)) if rng.random() < 0.7 else 64 * int(rng.integers(1, 5))
+        H = max(H, 8) // D * D or D
+        N = int(rng.choice([rng.integers(1, 40), rng.integers(40, 600), rng.integers(600, 2300)]))
+        lag = int(rng.integers(0, 6))
+        S = int(rng.integers(1, 700))
+        prec = int(rng.integers(0, 3))
+        literal = bool(rng.random() < 0.5)
+        shapes.append((N, D, H, lag, S, prec, literal))
+    return shapes
+
+
+@pytest.mark.parametrize("N,D,H,lag,S,prec,literal", _random_shapes(16, seed=20260101))
+def test_random_shapes_both_variants(N, D, H, lag, S, prec, literal):
+    # shapes nobody picked by hand: every kernel selection rule (tensor-core chain or not, resident encoder or not,
+    # sort width, ragged tiles) gets exercised in combinations
+    make = inputs.make_weights_literal if literal else inputs.make_weights
+    w = make(N, D, H, seed=N + H, fan_in_ref=32, bf16=(prec == 2))
+    trace = inputs.make_trace(N, lag + 3, seed=S, sigma=0.25)
+    gpu = binding.Cutoff(N, D, H, lag, S, precision=prec, seed=SEED + N, flags=binding.FLAG_LITERAL if literal else 0)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, lag, S, seed=SEED + N)
+    for x in trace:
+        gpu.push(x)
+        orc.push(x)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec] if prec else 2e-5)
+    assert_decision_close(gpu, orc.predict(), N)
