@@ -526,3 +526,55 @@ def test_random_shapes_both_variants(N, D, H, lag, S, prec, literal):
         orc.push(x)
     assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec] if prec else 2e-5)
     assert_decision_close(gpu, orc.predict(), N)
+
+
+@pytest.mark.parametrize("seed,literal,graph", [(1, False, False), (2, True, False), (3, False, True), (4, True, True)])
+def test_random_call_sequences(seed, literal, graph):
+    # pushes from host and device, decisions, save / restore, reset and reloaded weights in random order: the
+    # library's cached state (window, normaliser, per-slot projections, captured graph) must follow the oracle's
+    import copy
+    import torch
+    rng = np.random.default_rng(seed)
+    N, D, H, lag, S = 96, 8, 64, 2, 192
+    make = inputs.make_weights_literal if literal else inputs.make_weights
+    weights = [make(N, D, H, seed=s, fan_in_ref=32) for s in (11, 12)]
+    trace = inputs.make_trace(N, 80, seed=seed, sigma=0.25)
+    flags = (binding.FLAG_LITERAL if literal else 0) | (binding.FLAG_GRAPH if graph else 0)
+    gpu = binding.Cutoff(N, D, H, lag, S, seed=SEED, flags=flags)
+    gpu.load_weights(weights[0])
+    orc = O.CutoffOracle(weights[0], lag, S, seed=SEED)
+    saved = None
+    t = 0
+    decisions = 0
+    for _ in range(60):
+        op = rng.choice(["push", "push_dev", "predict", "step", "save", "restore", "reset", "weights"],
+                        p=[0.25, 0.1, 0.25, 0.15, 0.07, 0.07, 0.04, 0.07])
+        if op == "push":
+            gpu.push(trace[t]); orc.push(trace[t]); t += 1
+        elif op == "push_dev":
+            gpu.push(torch.from_numpy(trace[t]).cuda()); orc.push(trace[t]); t += 1
+        elif op in ("predict", "step"):
+            if op == "step":
+                res_g = gpu.step(trace[t]); orc.push(trace[t]); t += 1
+            else:
+                res_g = gpu.predict()
+            code_o, c_o, e_o, om_o = orc.predict()
+            assert res_g[0] == code_o
+            if code_o == O.WARMUP:
+                assert res_g[1] == N
+                continue
+            decisions += 1
+            e_g, _ = gpu.get_stats()
+            assert np.max(np.abs(e_g - e_o) / np.abs(e_o[-1])) <= TOL_E
+            top = np.sort(om_o[np.isfinite(om_o)])[-2:]
+            assert res_g[1] == c_o or (top[1] - top[0]) <= TOL_E * abs(top[1])
+        elif op == "save":
+            saved = (gpu.save_state(), copy.deepcopy(orc.history), orc.step)
+        elif op == "restore" and saved is not None:
+            gpu.restore_state(saved[0]); orc.history = copy.deepcopy(saved[1]); orc.step = saved[2]
+        elif op == "reset":
+            gpu.reset(); orc.reset()
+        elif op == "weights":
+            w = weights[int(rng.integers(0, 2))]
+            gpu.load_weights(w); orc.w = w
+    assert decisions >= 5
