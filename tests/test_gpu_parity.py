@@ -528,14 +528,15 @@ def test_random_shapes_both_variants(N, D, H, lag, S, prec, literal):
     assert_decision_close(gpu, orc.predict(), N)
 
 
-@pytest.mark.parametrize("seed,literal,graph", [(1, False, False), (2, True, False), (3, False, True), (4, True, True)])
-def test_random_call_sequences(seed, literal, graph):
+@pytest.mark.parametrize("seed,literal,graph,H", [(1, False, False, 64), (2, True, False, 64), (3, False, True, 64),
+                                                  (4, True, True, 64), (5, False, True, 320), (6, False, False, 512)])
+def test_random_call_sequences(seed, literal, graph, H):
     # pushes from host and device, decisions, save / restore, reset and reloaded weights in random order: the
     # library's cached state (window, normaliser, per-slot projections, captured graph) must follow the oracle's
     import copy
     import torch
     rng = np.random.default_rng(seed)
-    N, D, H, lag, S = 96, 8, 64, 2, 192
+    N, D, lag, S = 96, 8, 2, 192        # H = 320 and 512: the cluster recurrence of the encoder, also inside the graph
     make = inputs.make_weights_literal if literal else inputs.make_weights
     weights = [make(N, D, H, seed=s, fan_in_ref=32) for s in (11, 12)]
     trace = inputs.make_trace(N, 80, seed=seed, sigma=0.25)
