@@ -162,6 +162,13 @@ int cutoff_fetch(cutoff_ctx* ctx, int32_t* c_out);
  * Returns what cutoff_predict returns.  Errors: BAD_ARG, BAD_VALUE, STATE, CUDA, TIMEOUT. */
 int cutoff_step(cutoff_ctx* ctx, const float* runtimes_sec, int32_t* c_out);
 
+/* The same with the run-times already on the context's device (N floats): with CUTOFF_FLAG_GRAPH one
+ * device-to-device copy into the library's landing buffer, then a replay of the captured push + decision.
+ * The values are checked on the GPU: a value that is not finite or not > 0 leaves the window and the
+ * decision counter as they were and returns BAD_VALUE after the replay.
+ * Errors: BAD_ARG, BAD_VALUE, STATE, CUDA, TIMEOUT. */
+int cutoff_step_device(cutoff_ctx* ctx, const float* runtimes_sec_device, int32_t* c_out);
+
 /* Results of the last completed decision.  Either pointer may be NULL.
  * exp_order_stats_sec (host, N floats): E[x~_(j)] in seconds, ascending.
  * omega_per_sec (host, N floats): Omega(c) = c / E[x~_(c)]; -inf where E <= 0.

@@ -27,7 +27,7 @@ BLOB_MAGIC = 0x31465443
 
 EXPORTS = (
     "cutoff_create", "cutoff_destroy", "cutoff_load_weights", "cutoff_push", "cutoff_push_async",
-    "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_step", "cutoff_get_stats",
+    "cutoff_predict", "cutoff_predict_async", "cutoff_fetch", "cutoff_step", "cutoff_step_device", "cutoff_get_stats",
     "cutoff_get_order_stat_std", "cutoff_get_partial_sums", "cutoff_decide_from_sums", "cutoff_reset", "cutoff_save_state",
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
@@ -74,6 +74,7 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_predict_async": (C.c_int, [vp]),
         "cutoff_fetch": (C.c_int, [vp, i32p]),
         "cutoff_step": (C.c_int, [vp, vp, i32p]),
+        "cutoff_step_device": (C.c_int, [vp, vp, i32p]),
         "cutoff_get_stats": (C.c_int, [vp, vp, vp]),
         "cutoff_get_order_stat_std": (C.c_int, [vp, vp]),
         "cutoff_get_partial_sums": (C.c_int, [vp, vp]),
@@ -214,6 +215,14 @@ class Cutoff:
             raise ValueError("expected N run-times")
         c = C.c_int32(0)
         rc = self._check(self._lib.cutoff_step(self._h, a.ctypes.data, C.byref(c)), "cutoff_step")
+        return rc, c.value
+
+    def step_device(self, runtimes_sec_device):
+        """As step(), with the run-times in a contiguous CUDA tensor of N fp32 values; returns (code, c)."""
+        if tuple(runtimes_sec_device.shape) != (self.N,) or not runtimes_sec_device.is_cuda or not runtimes_sec_device.is_contiguous():
+            raise ValueError("expected a contiguous CUDA tensor of N fp32 run-times")
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_step_device(self._h, runtimes_sec_device.data_ptr(), C.byref(c)), "cutoff_step_device")
         return rc, c.value
 
     def get_stats(self):

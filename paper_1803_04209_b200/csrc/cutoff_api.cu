@@ -103,6 +103,8 @@ struct cutoff_ctx {
 
     cudaGraph_t graph = nullptr;            // captured push + decision (CUTOFF_FLAG_GRAPH)
     cudaGraphExec_t graph_exec = nullptr;
+    cudaGraph_t graph_dev = nullptr;        // the same without the host-to-device copy (cutoff_step_device)
+    cudaGraphExec_t graph_dev_exec = nullptr;
     int graph_kernels = 0;                  // kernels one replay launches
     bool decided_once = false;              // a decision has run outside capture (function attributes are set)
 
@@ -164,6 +166,8 @@ void free_all(cutoff_ctx* c) {
     if (c->owns_stream && c->stream) cudaStreamDestroy(c->stream);
     if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
     if (c->graph) cudaGraphDestroy(c->graph);
+    if (c->graph_dev_exec) cudaGraphExecDestroy(c->graph_dev_exec);
+    if (c->graph_dev) cudaGraphDestroy(c->graph_dev);
     if (c->ev_created)
         for (auto& row : c->ev)
             for (auto& e : row)
@@ -1108,11 +1112,11 @@ int cutoff_predict(cutoff_ctx* c, int32_t* c_out) {
 // Capture "land the staged run-times, push, decide, read back the state" once; replays need no
 // changing argument because the window position, the normaliser and the decision counter live
 // in device memory.
-static int build_graph(cutoff_ctx* c) {
+static int build_graph(cutoff_ctx* c, bool with_host_copy) {
     refresh_projections(c);                        // not part of the graph: replays only project the vector they push
     const int64_t launches_before = c->launches;
     CU_CHECK(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-    cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, cudaMemcpyHostToDevice, c->stream);
+    if (with_host_copy) cudaMemcpyAsync(c->d_stage, c->h_stage, sizeof(float) * c->N, cudaMemcpyHostToDevice, c->stream);
     k_push<<<1, kPushThreads, 0, c->stream>>>(c->d_stage, c->d_ring, c->d_state, c->N, c->W);
     c->launches += 1;
     launch_projection(c, true);
@@ -1130,8 +1134,13 @@ static int build_graph(cutoff_ctx* c) {
         cudaGetLastError();
         return CUTOFF_ERR_CUDA;
     }
-    c->graph = g;
-    CU_CHECK(c, cudaGraphInstantiate(&c->graph_exec, c->graph, 0));
+    if (with_host_copy) {
+        c->graph = g;
+        CU_CHECK(c, cudaGraphInstantiate(&c->graph_exec, c->graph, 0));
+    } else {
+        c->graph_dev = g;
+        CU_CHECK(c, cudaGraphInstantiate(&c->graph_dev_exec, c->graph_dev, 0));
+    }
     return CUTOFF_OK;
 }
 
@@ -1150,7 +1159,7 @@ int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
     CU_CHECK(c, cudaSetDevice(c->cfg.device));
     if (!c->graph_exec) {
         CU_CHECK(c, cudaStreamSynchronize(c->stream));
-        const int rc = build_graph(c);
+        const int rc = build_graph(c, true);
         if (rc) return rc;
     }
     std::memcpy(c->h_stage, runtimes_sec, sizeof(float) * c->N);     // the stream is idle: every call ends synchronised
@@ -1158,6 +1167,45 @@ int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
     CU_CHECK(c, cudaGraphLaunch(c->graph_exec, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     c->launches += c->graph_kernels;
+    c->pushes += 1;
+    c->draws_valid = c->n_chunks == 1;
+    if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
+    c->have_result = true;
+    *c_out = c->h_state->c_star;
+    return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
+}
+
+int cutoff_step_device(cutoff_ctx* c, const float* runtimes_sec_device, int32_t* c_out) {
+    if (!c || !runtimes_sec_device || !c_out) return CUTOFF_ERR_BAD_ARG;
+    if (!c->weights_loaded || c->pending) return CUTOFF_ERR_STATE;
+    const bool replay = (c->cfg.flags & CUTOFF_FLAG_GRAPH) && c->decided_once &&
+                        c->pushes + 1 >= static_cast<uint32_t>(c->W);
+    if (!replay) {
+        const int rc = cutoff_push(c, runtimes_sec_device, 1, nullptr);
+        if (rc < 0) return rc;
+        return cutoff_predict(c, c_out);
+    }
+    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (!c->graph_dev_exec) {
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));
+        const int rc = build_graph(c, false);
+        if (rc) return rc;
+    }
+    refresh_projections(c);
+    CU_CHECK(c, cudaMemcpyAsync(c->d_stage, runtimes_sec_device, sizeof(float) * c->N, cudaMemcpyDeviceToDevice, c->stream));
+    CU_CHECK(c, cudaGraphLaunch(c->graph_dev_exec, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    c->launches += c->graph_kernels;
+    if (c->h_state->error_flags & kErrBadValue) {
+        // the push kernel left the window untouched, but the decision that followed it ran on the old window and
+        // advanced the decision counter: put the counter back, clear the flag, report the bad value
+        const uint32_t step_before = c->h_state->step - 1u;
+        CU_CHECK(c, cudaMemcpyAsync(&c->d_state->step, &step_before, sizeof(uint32_t), cudaMemcpyHostToDevice, c->stream));
+        CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
+        CU_CHECK(c, cudaStreamSynchronize(c->stream));
+        c->draws_valid = false;
+        return CUTOFF_ERR_BAD_VALUE;
+    }
     c->pushes += 1;
     c->draws_valid = c->n_chunks == 1;
     if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
@@ -1288,7 +1336,7 @@ int cutoff_set_option(cutoff_ctx* c, const char* name, int64_t value) {
     if (std::strcmp(name, "order_stat_std") == 0) {
         if (value != 0 && value != 1) return CUTOFF_ERR_BAD_ARG;
         if (value && c->cfg.total_samples > 0 && c->cfg.total_samples != c->S) return CUTOFF_ERR_UNSUPPORTED;
-        if (c->graph_exec) return CUTOFF_ERR_STATE;                // the captured graph has the other sort kernel in it
+        if (c->graph_exec || c->graph_dev_exec) return CUTOFF_ERR_STATE;   // the captured graph has the other sort kernel in it
         c->want_std = value != 0;
         return CUTOFF_OK;
     }

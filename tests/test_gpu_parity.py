@@ -579,3 +579,35 @@ def test_random_call_sequences(seed, literal, graph, H):
             w = weights[int(rng.integers(0, 2))]
             gpu.load_weights(w); orc.w = w
     assert decisions >= 5
+
+
+def test_step_device_equals_step_and_rejects_bad_values():
+    # run-times that already sit on the GPU: same decisions as the host call, with and without the graph
+    import torch
+    wl = inputs.WORKLOADS["stream"]
+    S = 384
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, wl.window + 10)
+    dev = torch.from_numpy(trace).cuda()
+    host_ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED, flags=binding.FLAG_GRAPH)
+    dev_ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED, flags=binding.FLAG_GRAPH)
+    plain_ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED)
+    for ctx in (host_ctx, dev_ctx, plain_ctx):
+        ctx.load_weights(w)
+    for t in range(trace.shape[0]):
+        a, b, c = host_ctx.step(trace[t]), dev_ctx.step_device(dev[t]), plain_ctx.step_device(dev[t])
+        assert a == b == c
+        if a[0] == binding.OK:
+            assert np.array_equal(host_ctx.get_stats()[0], dev_ctx.get_stats()[0])
+            assert np.array_equal(host_ctx.get_stats()[0], plain_ctx.get_stats()[0])
+    # a bad value inside a replay: reported, and nothing has moved (window, decision counter)
+    bad = dev[3].clone()
+    bad[17] = -1.0
+    for ctx in (dev_ctx, plain_ctx):
+        with pytest.raises(binding.CutoffError) as e:
+            ctx.step_device(bad)
+        assert e.value.code == binding.ERR_BAD_VALUE
+    nxt = trace[5]
+    a, b, c = host_ctx.step(nxt), dev_ctx.step_device(torch.from_numpy(nxt).cuda()), plain_ctx.step_device(torch.from_numpy(nxt).cuda())
+    assert a == b == c
+    assert np.array_equal(host_ctx.get_stats()[0], dev_ctx.get_stats()[0])
