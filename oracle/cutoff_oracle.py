@@ -36,10 +36,9 @@ vectors, against a second big-integer implementation and against its own
 inverse; Box-Muller against N(0,1) moments and a KS test; the sort/mean/argmax
 tail against the iid-normal order-statistic integral of Section 3.1.1, the
 worked example of Section 4.1 and brute force; the networks against
-linear-Gaussian closed forms and special cases.  The general nonlinear
-networks (ReLU / tanh with dense random weights) have no closed form:
-**parity unpinned** for ``encoder`` and ``guide_chain`` beyond those special
-cases.
+linear-Gaussian closed forms and special cases; ``encoder`` and ``guide_chain``
+with dense, non-symmetric weights, non-zero initial states and noise against
+scalar loops written element by element from the guide equations.
 
 Model variants.  "compact": transition and emission are one-hidden-layer ReLU
 MLPs with a (mean, log-variance) head (``transition`` / ``emission``).

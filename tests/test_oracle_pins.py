@@ -338,6 +338,97 @@ def test_guide_chain_noise_free_scalar_recursion():
     assert np.allclose(z, want, rtol=1e-13)
 
 
+def test_encoder_against_scalar_loops_dense_nonsymmetric_recurrence():
+    # h_left(t) = relu(Wxf x_t + Whf h_left(t-1) + bf) from a0, h_right(t) likewise backwards from b0
+    # (Section 3.1.3, guide): written out element by element, with dense non-symmetric recurrent matrices,
+    # non-zero initial states and several window positions, so that a transposed Whf / Whb, a swapped
+    # direction or a dropped initial state shows.
+    N, H, W = 5, 4, 4
+    rng = np.random.default_rng(21)
+    w = inputs.make_weights(N, 3, H, seed=12, std=0.6, offsets=False)
+    w["a0"] = rng.uniform(0.2, 1.0, size=H).astype(np.float32)
+    w["b0"] = rng.uniform(0.2, 1.0, size=H).astype(np.float32)
+    assert not np.allclose(w["Whf"], w["Whf"].T) and not np.allclose(w["Whb"], w["Whb"].T)
+    xhat = rng.uniform(0.1, 1.2, size=(W, N))
+    a, b = O.encoder(xhat, w)
+    f = {k: v.astype(np.float64) for k, v in w.items()}
+    state = [float(v) for v in f["a0"]]
+    active = 0
+    for t in range(W):
+        new = []
+        for i in range(H):
+            pre = f["bf"][i]
+            for j in range(N):
+                pre += f["Wxf"][i][j] * xhat[t][j]
+            for j in range(H):
+                pre += f["Whf"][i][j] * state[j]
+            new.append(max(pre, 0.0))
+        state = new
+        active += sum(v > 0 for v in new)
+        for i in range(H):
+            assert abs(a[t][i] - state[i]) < 1e-12
+    state = [float(v) for v in f["b0"]]
+    for t in range(W - 1, -1, -1):
+        new = []
+        for i in range(H):
+            pre = f["bb"][i]
+            for j in range(N):
+                pre += f["Wxb"][i][j] * xhat[t][j]
+            for j in range(H):
+                pre += f["Whb"][i][j] * state[j]
+            new.append(max(pre, 0.0))
+        state = new
+        active += sum(v > 0 for v in new)
+        for i in range(H):
+            assert abs(b[t][i] - state[i]) < 1e-12
+    assert active >= W * H // 2          # the case is not vacuous: most units carry state forward
+    # the pin has teeth: the same loops against a transposed recurrence disagree
+    wt = dict(w); wt["Whf"] = w["Whf"].T.copy()
+    assert np.max(np.abs(O.encoder(xhat, wt)[0] - a)) > 1e-3
+
+
+def test_guide_chain_against_scalar_loops_dense_weights_with_noise():
+    # z_t = mu + sigma * eps,  h_out = (tanh(Wz z_{t-1} + bz) + h_left(t) + h_right(t)) / 3,
+    # mu = Wmu h_out + bmu,  sigma = softplus(Wsig mu + bsig)   (Section 3.1.3, guide), element by element:
+    # dense Wz feeding dense Wmu feeding dense Wsig over three steps, non-zero z0, noise on.
+    D, H, W, S = 3, 5, 3, 4
+    rng = np.random.default_rng(22)
+    w = inputs.make_weights(4, D, H, seed=13, std=0.8, offsets=False)
+    w["z0"] = rng.normal(size=D).astype(np.float32)
+    a = np.abs(rng.normal(size=(W, H)))
+    b = np.abs(rng.normal(size=(W, H)))
+    eps = rng.standard_normal((S, W, D))
+    got = O.guide_chain(a, b, w, eps)
+    f = {k: v.astype(np.float64) for k, v in w.items()}
+    for k in range(S):
+        z = [float(v) for v in f["z0"]]
+        for t in range(W):
+            h_out = []
+            for i in range(H):
+                pre = f["bz"][i]
+                for d in range(D):
+                    pre += f["Wz"][i][d] * z[d]
+                h_out.append((math.tanh(pre) + a[t][i] + b[t][i]) / 3.0)
+            mu = []
+            for d in range(D):
+                acc = f["bmu"][d]
+                for i in range(H):
+                    acc += f["Wmu"][d][i] * h_out[i]
+                mu.append(acc)
+            z = []
+            for d in range(D):
+                pre = f["bsig"][d]
+                for e in range(D):
+                    pre += f["Wsig"][d][e] * mu[e]
+                z.append(mu[d] + math.log1p(math.exp(pre)) * eps[k][t][d])
+        for d in range(D):
+            assert abs(got[k][d] - z[d]) < 1e-12
+    # teeth: a transposed Wsig, or the window's encodings taken in reverse order, change the result
+    wt = dict(w); wt["Wsig"] = w["Wsig"].T.copy()
+    assert np.max(np.abs(O.guide_chain(a, b, wt, eps) - got)) > 1e-3
+    assert np.max(np.abs(O.guide_chain(a[::-1], b[::-1], w, eps) - got)) > 1e-3
+
+
 def test_guide_head_orientation():
     # Wz = 0: h_out is the same for every sample, so mu = Wmu h + bmu and sigma = softplus(Wsig mu + bsig)
     D, H, S = 3, 5, 1 << 15
