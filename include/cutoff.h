@@ -37,6 +37,8 @@
  *     Caller pointers are borrowed for the duration of the call only.
  *   - A context owns all device memory it allocates and is bound to one
  *     device and one stream.  It is not thread-safe.
+ *   - Every entry point makes the context's device current while it runs and
+ *     puts the caller's current device back before it returns.
  *   - Nothing here throws, aborts or calls exit().
  */
 #ifndef CUTOFF_H_
@@ -96,7 +98,8 @@ typedef struct {
     uint64_t seed;              /* Philox key                                                      */
 } cutoff_config;
 
-/* Create a context: validates cfg, selects the device, allocates all device memory.
+/* Create a context: validates cfg, allocates all device memory on cfg->device, and tells that device
+ * which of the library's kernels need large shared memory (so contexts on several GPUs can live in one process).
  * out (host) receives the handle.  Errors: BAD_ARG, UNSUPPORTED, NOMEM, CUDA. */
 int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg);
 
@@ -188,6 +191,24 @@ int cutoff_get_order_stat_std(cutoff_ctx* ctx, float* std_sec);
 int cutoff_get_partial_sums(cutoff_ctx* ctx, double* sums);
 int cutoff_decide_from_sums(cutoff_ctx* ctx, const double* sums, int32_t* c_out);
 
+/* The same exchange with nothing passing through the host, for several contexts (one per GPU) that share a
+ * decision (the K samples of the predictive approximation after Eq. 4 are independent, so they split):
+ *   cutoff_predict_partial_async   enqueue this context's part of the decision up to the per-position sums of its
+ *                                  sorted samples and return at once; no argmax, the decision counter stays.
+ *                                  Returns OK, or WARMUP (fewer than lag+1 vectors: nothing enqueued, c = N).
+ *   cutoff_partial_sums_device     *sums_device = the context's own N doubles (device memory; valid until
+ *                                  cutoff_destroy) that hold those sums once the enqueued work is done.  They may
+ *                                  be all-reduced in place by work enqueued on the context's stream.
+ *   cutoff_decide_from_device_sums finish the decision from sums over all total_samples samples
+ *                                  (sums_device: device, N doubles; may be the context's own array), advance
+ *                                  the decision counter if the sums came from cutoff_predict_partial_async,
+ *                                  wait, and return what cutoff_predict returns.
+ * Errors: BAD_ARG, STATE (weights missing, a decision already in flight, too few observations), BAD_VALUE (an
+ * asynchronous push before it carried a bad value), CUDA, TIMEOUT. */
+int cutoff_predict_partial_async(cutoff_ctx* ctx);
+int cutoff_partial_sums_device(cutoff_ctx* ctx, double** sums_device);
+int cutoff_decide_from_device_sums(cutoff_ctx* ctx, const double* sums_device, int32_t* c_out);
+
 /* Forget all observations and restart the decision counter. */
 int cutoff_reset(cutoff_ctx* ctx);
 
@@ -209,6 +230,12 @@ const char* cutoff_last_error(cutoff_ctx* ctx);
  * cutoff_stage_name names stage i.  cutoff_launch_count returns the number of kernels this
  * context has launched since it was created. */
 int cutoff_set_timing(cutoff_ctx* ctx, int on);
+/* cutoff_measure_pipe_rates: the issue rates that bound the sort (Section 3.1.1, last paragraph) and the
+ * per-sample chain on this device, measured by a short micro-benchmark (about 10 ms): rates_out (host,
+ * 3 floats) = warp-instructions per clock per SM of fp32 min/max, of warp shuffles and of fp32 fused
+ * multiply-adds, each from 32 warps per SM running independent chains.  Allocates and frees a few KB of
+ * device memory, synchronises the device.  Errors: BAD_ARG, NOMEM, CUDA. */
+int cutoff_measure_pipe_rates(int device, float* rates_out);
 int cutoff_get_timing(cutoff_ctx* ctx, float* ms, int cap);
 const char* cutoff_stage_name(int i);
 int64_t cutoff_launch_count(cutoff_ctx* ctx);
@@ -241,6 +268,11 @@ int cutoff_debug_samples(cutoff_ctx* ctx, int64_t k0, int64_t count, float* x_ou
 int cutoff_debug_window(cutoff_ctx* ctx, float* window_out);
 int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n,
                       float* keys_out, int32_t* perm_out);
+/* cutoff_debug_sort_values: the same networks in the instantiation the decision itself runs (plain
+ * fp32 keys, rows padded with +infinity), the sorted rows returned instead of summed (Section 3.1.1,
+ * last paragraph: "sort").  rows (host, n_rows*n floats, any finite values, +-0 and +infinity
+ * included) -> keys_out (host, n_rows*n floats, each row ascending).  n <= 4096. */
+int cutoff_debug_sort_values(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n, float* keys_out);
 
 /* ---- allocation-free entry point ---------------------------------------------------------------
  * The paper has no counterpart for this call.  It serves programs that may not allocate device
@@ -255,13 +287,16 @@ int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_
  * Dividing by n_rows gives the Monte-Carlo expected order statistics of Section 3.1.1.
  *   device    CUDA device ordinal (0..63) that owns x, sums and stream
  *   x         device, n_rows x ldx floats, row-major; entries beyond n in a row are ignored
- *   n_rows    1 .. 2^31-1;   n  1 .. CUTOFF_STATIC_MAX_N;   ldx >= n
+ *   n_rows    1 .. CUTOFF_STATIC_MAX_ROWS;   n  1 .. CUTOFF_STATIC_MAX_N;   ldx >= n
  *   sums      device, n doubles, overwritten
+ * Accuracy: the rows go through in blocks of 131072; inside a block a warp adds at most 64 sorted rows in
+ * single precision, everything above that is added in double, so the error of a sum does not grow with
+ * n_rows beyond that of 64 single-precision additions (about 4e-6 relative to the largest partial sum).
  *   stream    cudaStream_t to run on (NULL = default stream); the call only enqueues work
  * The call performs no cudaMalloc, cudaFree or other allocating routine.  Its only scratch is a
  * fixed array of CUTOFF_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that
  * loads the library holds that much memory until the process exits.  n above the limit returns
- * CUTOFF_ERR_TOO_LARGE and does nothing.
+ * CUTOFF_ERR_TOO_LARGE and does nothing; n_rows above CUTOFF_STATIC_MAX_ROWS returns BAD_ARG.
  * The first call on a device looks up the array's device address (a one-time set-up step that
  * loads the library's code on that device); make that first call before starting any stream
  * capture.  All calls on a device share the one array, and it keeps what the last call left in
@@ -270,6 +305,7 @@ int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_
  * Issue them on one stream, or order them with events.  Not thread-safe with respect to its
  * first call on a device.  Errors: BAD_ARG, TOO_LARGE, CUDA. */
 #define CUTOFF_STATIC_MAX_N 1024
+#define CUTOFF_STATIC_MAX_ROWS (1 << 24)
 #define CUTOFF_STATIC_SCRATCH_BYTES (256 * 1024 * 4)
 int cutoff_sorted_row_sums_static(int device, const float* x, int64_t n_rows, int32_t n, int32_t ldx,
                                   double* sums, void* stream);

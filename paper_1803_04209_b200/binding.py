@@ -32,6 +32,8 @@ EXPORTS = (
     "cutoff_restore_state", "cutoff_strerror", "cutoff_last_error", "cutoff_set_timing",
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
     "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
+    "cutoff_debug_sort_values", "cutoff_predict_partial_async", "cutoff_partial_sums_device",
+    "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates",
     "cutoff_sorted_row_sums_static",
 )
 
@@ -94,6 +96,11 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_debug_samples": (C.c_int, [vp, C.c_int64, C.c_int64, vp]),
         "cutoff_debug_window": (C.c_int, [vp, vp]),
         "cutoff_debug_sort": (C.c_int, [vp, vp, C.c_int64, C.c_int32, vp, vp]),
+        "cutoff_debug_sort_values": (C.c_int, [vp, vp, C.c_int64, C.c_int32, vp]),
+        "cutoff_predict_partial_async": (C.c_int, [vp]),
+        "cutoff_partial_sums_device": (C.c_int, [vp, C.POINTER(vp)]),
+        "cutoff_decide_from_device_sums": (C.c_int, [vp, vp, i32p]),
+        "cutoff_measure_pipe_rates": (C.c_int, [C.c_int, f32p]),
         "cutoff_sorted_row_sums_static": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -251,6 +258,36 @@ class Cutoff:
         rc = self._check(self._lib.cutoff_decide_from_sums(self._h, s.ctypes.data, C.byref(c)), "cutoff_decide_from_sums")
         return rc, c.value
 
+    def predict_partial_async(self) -> int:
+        """Enqueue this context's share of a decision up to the per-position sums; returns OK or WARMUP."""
+        return self._check(self._lib.cutoff_predict_partial_async(self._h), "cutoff_predict_partial_async")
+
+    def partial_sums_device_ptr(self) -> int:
+        """Device address of the context's N doubles (the per-position sums)."""
+        p = C.c_void_p()
+        self._check(self._lib.cutoff_partial_sums_device(self._h, C.byref(p)), "cutoff_partial_sums_device")
+        return p.value
+
+    def partial_sums_tensor(self):
+        """The same array as a torch CUDA tensor that aliases the library's memory (no copy)."""
+        import torch
+
+        class _Alias:
+            pass
+        a = _Alias()
+        a.__cuda_array_interface__ = {"shape": (self.N,), "typestr": "<f8", "data": (self.partial_sums_device_ptr(), False),
+                                      "version": 2}
+        return torch.as_tensor(a, device=torch.device("cuda", self.cfg.device))
+
+    def decide_from_device_sums(self, sums_device):
+        """sums_device: a CUDA tensor of N doubles (possibly partial_sums_tensor()); returns (code, c)."""
+        if tuple(sums_device.shape) != (self.N,) or not sums_device.is_cuda or sums_device.element_size() != 8:
+            raise ValueError("expected a CUDA tensor of N doubles")
+        c = C.c_int32(0)
+        rc = self._check(self._lib.cutoff_decide_from_device_sums(self._h, sums_device.data_ptr(), C.byref(c)),
+                         "cutoff_decide_from_device_sums")
+        return rc, c.value
+
     def reset(self):
         self._check(self._lib.cutoff_reset(self._h), "cutoff_reset")
 
@@ -300,6 +337,14 @@ class Cutoff:
                                                 perm.ctypes.data), "cutoff_debug_sort")
         return keys, perm
 
+    def debug_sort_values(self, rows: np.ndarray) -> np.ndarray:
+        """Rows sorted ascending by the fp32 network of the decision path."""
+        r = np.ascontiguousarray(rows, dtype=np.float32)
+        keys = np.empty_like(r)
+        self._check(self._lib.cutoff_debug_sort_values(self._h, r.ctypes.data, r.shape[0], r.shape[1], keys.ctypes.data),
+                    "cutoff_debug_sort_values")
+        return keys
+
 
 def debug_normals(seed: int, step: int, stream: int, k0: int, count: int, n_elems: int, device: int = 0):
     """(normals[count, n_elems] fp32, words[count, ceil(n_elems/4), 4] uint32) from the GPU generator."""
@@ -311,6 +356,16 @@ def debug_normals(seed: int, step: int, stream: int, k0: int, count: int, n_elem
     if rc < 0:
         raise CutoffError(rc, "cutoff_debug_normals")
     return normals, words
+
+
+def measure_pipe_rates(device: int = 0) -> dict:
+    """Measured issue rates (warp-instructions per clock per SM) of fp32 min/max, shuffles and fp32 FMA."""
+    lib = load_library()
+    out = (C.c_float * 3)()
+    rc = lib.cutoff_measure_pipe_rates(device, out)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_measure_pipe_rates")
+    return {"minmax": float(out[0]), "shuffle": float(out[1]), "fma": float(out[2])}
 
 
 def sorted_row_sums_static(x, sums, n: int | None = None, stream: int | None = None) -> int:

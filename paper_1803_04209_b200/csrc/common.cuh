@@ -13,7 +13,7 @@ struct DevState {
     float inv_scale;
     uint32_t push_count;    // vectors pushed since reset
     uint32_t step;          // decisions made since reset (addresses the noise)
-    int32_t error_flags;    // bit 0: a pushed value was not finite or not > 0; bit 1: device wait timed out
+    int32_t error_flags;    // bit 0: a pushed value was not finite or not > 0; bit 1: device wait timed out; bit 2: all workers censored
     int32_t c_star;         // last decision
     int32_t code;           // 0 ok, 2 degenerate
     uint32_t ticket;        // CTAs that have finished their column sums (self-resetting)
@@ -21,6 +21,7 @@ struct DevState {
 
 constexpr int kErrBadValue = 1;
 constexpr int kErrTimeout = 2;
+constexpr int kErrNoFinisher = 4;   // a censored push in which every worker was censored
 
 // Model dimensions and device pointers handed to the kernels by value.
 struct ModelDev {

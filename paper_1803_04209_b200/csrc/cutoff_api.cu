@@ -17,6 +17,7 @@
 #include "kernels_literal.cuh"
 #include "gemm_tc.cuh"
 #include "chain_tc_literal.cuh"
+#include "pipe_rates.cuh"
 
 using namespace cutoff;
 
@@ -94,6 +95,7 @@ struct cutoff_ctx {
     bool pending = false;           // a decision is enqueued and not yet fetched
     bool pending_warmup = false;
     bool have_result = false;
+    bool partial_pending = false;   // the sums of a decision are enqueued, its argmax (and counter step) still to come
 
     bool timing = false;
     cudaEvent_t ev[kNumStages + 1][kMaxChunks]{};   // per chunk, stage boundaries
@@ -122,6 +124,26 @@ namespace {
             return err__ == cudaErrorMemoryAllocation ? CUTOFF_ERR_NOMEM : CUTOFF_ERR_CUDA;          \
         }                                                                                            \
     } while (0)
+
+// Makes the context's device current for the duration of an entry point and puts the caller's
+// current device back on exit.
+struct DeviceGuard {
+    int prev = -1;
+    bool changed = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int device) {
+        if (cudaGetDevice(&prev) != cudaSuccess) prev = -1;
+        if (prev != device) {
+            err = cudaSetDevice(device);
+            changed = err == cudaSuccess;
+        }
+    }
+    ~DeviceGuard() {
+        if (changed && prev >= 0) cudaSetDevice(prev);
+    }
+    DeviceGuard(const DeviceGuard&) = delete;
+    DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
 
 std::vector<TensorSpec> tensor_specs(size_t N, size_t D, size_t H) {
     return {
@@ -193,12 +215,7 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
 
 template <int E, bool SQ>
 void launch_sort_warp_sq(cutoff_ctx* c, int count, float* partial) {
-    static bool attr_set = false;
     const size_t smem = sort_tma_smem_bytes<E>(c->ldx);
-    if (!attr_set) {
-        cudaFuncSetAttribute(k_sort_sum_tma<E, SQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024);
-        attr_set = true;
-    }
     k_sort_sum_tma<E, SQ><<<c->sort_grid, kSortWarps * 32, smem, c->stream>>>(
         c->d_x, c->ldx, c->N, count, partial, partial + static_cast<size_t>(kPartialRows) * c->N, c->d_state);
 }
@@ -234,12 +251,6 @@ int launch_sort(cutoff_ctx* c, int count, float* partial) {
 
 template <int D>
 void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(k_chain<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        cudaFuncSetAttribute(k_chain_resident<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        attr_set = true;
-    }
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     const int round_v = c->cfg.precision != CUTOFF_PRECISION_FP32;
     const size_t resident = chain_resident_smem_floats(c->D, c->H, c->W) * sizeof(float);
@@ -257,11 +268,6 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
 }
 
 void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_chain_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        attr_set = true;
-    }
     tc::ChainTcArgs a;
     const ModelDev& m = c->m;
     a.image = c->d_chain_image;
@@ -276,11 +282,6 @@ void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
 }
 
 void launch_chain_tc32(cutoff_ctx* c, uint32_t sample_base, int count) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_chain_tc32, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        attr_set = true;
-    }
     tc::ChainTc32Args a;
     const ModelDev& m = c->m;
     a.image = c->d_chain_image;
@@ -296,11 +297,6 @@ void launch_chain_tc32(cutoff_ctx* c, uint32_t sample_base, int count) {
 
 template <int D>
 void launch_chain_literal_t(cutoff_ctx* c, uint32_t sample_base, int count) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(k_chain_literal<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-        attr_set = true;
-    }
     const NoiseKey key{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     const size_t smem = chain_smem_floats(c->D, c->H, c->W) * sizeof(float);
     k_chain_literal<D><<<ceil_div(count, ChainShape<D>::kSamplesPerCta), ChainShape<D>::kThreads, smem, c->stream>>>(
@@ -308,11 +304,6 @@ void launch_chain_literal_t(cutoff_ctx* c, uint32_t sample_base, int count) {
 }
 
 void launch_chain_tc_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_chain_tc_literal, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-        attr_set = true;
-    }
     tc::ChainTclArgs a;
     const ModelDev& m = c->m;
     const LiteralDev& l = c->lit;
@@ -384,11 +375,6 @@ int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t r
 }
 
 void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_emit_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
-        attr_set = true;
-    }
     tc::EmitArgs a;
     a.b4 = c->m.b4; a.x = c->d_x; a.st = c->d_state;
     a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
@@ -401,11 +387,6 @@ void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
 
 // Literal emission (Section 3.1.3): I = u Wi2^T + bi2, r = relu(I Wj1^T + bj1), x = I + softplus(r Wj2^T + bj2) * eps.
 void launch_gemm_relu_tc(cutoff_ctx* c, const CUtensorMap& map_a, const CUtensorMap& map_b, const tc::GemmTcArgs& a) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(tc::k_gemm_relu_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kSmemBytes));
-        attr_set = true;
-    }
     const int tiles = ceil_div(a.Nout, tc::kGemmBN) * ceil_div(a.M, tc::kBM);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     tc::k_gemm_relu_tc<<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(map_a, map_b, a);
@@ -421,11 +402,6 @@ void launch_emission_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
         a.st = c->d_state; a.M = count; a.bias = c->d_M + static_cast<size_t>(c->H) * c->H; a.out = c->d_r;
         a.ld_out = c->H; a.Nout = c->H; a.K = c->H;
         launch_gemm_relu_tc(c, c->map_v, c->map_M, a);
-        static bool attr_set = false;
-        if (!attr_set) {
-            cudaFuncSetAttribute(tc::k_emit_dual_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(tc::kDualSmemBytes));
-            attr_set = true;
-        }
         tc::EmitDualArgs e;
         e.bias_mean = l.bi2; e.bias_scale = l.bj2; e.x = c->d_x; e.st = c->d_state; e.key = key;
         e.sample_base = sample_base; e.count = count; e.N = c->N; e.H = c->H; e.ldx = c->ldx;
@@ -460,11 +436,6 @@ void launch_emission(cutoff_ctx* c, uint32_t sample_base, int count) {
 
 template <int HQ>
 void launch_rnn_resident(cutoff_ctx* c) {
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaFuncSetAttribute(k_enc_rnn_resident<HQ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_set = true;
-    }
     const size_t smem = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float);
     k_enc_rnn_resident<HQ><<<2, 16 * HQ, smem, c->stream>>>(c->m, c->d_WhR, c->d_proj, c->d_state, c->d_hlr);
 }
@@ -494,11 +465,6 @@ void launch_encoder(cutoff_ctx* c) {
             const size_t cluster_smem = enc_rnn_cluster_smem_floats(c->H, c->W) * sizeof(float);
             if (!fits && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024) {
                 // the matrix of a direction split over a cluster of 8 CTAs
-                static bool attr_set = false;
-                if (!attr_set) {
-                    cudaFuncSetAttribute(k_enc_rnn_cluster, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-                    attr_set = true;
-                }
                 k_enc_rnn_cluster<<<2 * kRnnClusterSize, c->H, cluster_smem, c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
             } else {
                 k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
@@ -516,8 +482,9 @@ int ensure_events(cutoff_ctx* c) {
     return CUTOFF_OK;
 }
 
-// Enqueue one decision's kernels.  advance = 1 for a real decision, 0 for the debug hook.
-int enqueue_decision(cutoff_ctx* c) {
+// Enqueue one decision's kernels.  decide = false stops after the per-position sums (a context that holds
+// only part of a decision's samples: the argmax follows once the sums of all parts are added).
+int enqueue_decision(cutoff_ctx* c, bool decide = true) {
     const bool timed = c->timing;
     if (timed) {
         const int rc = ensure_events(c);
@@ -544,7 +511,7 @@ int enqueue_decision(cutoff_ctx* c) {
                                                                          c->d_sums, 1.0 / static_cast<double>(total),
                                                                          c->d_state, c->d_E, c->d_omega,
                                                                          c->want_std ? c->d_partial + static_cast<size_t>(kPartialRows) * c->N : nullptr,
-                                                                         c->d_std);
+                                                                         c->d_std, decide ? 1 : 0);
     c->have_std = c->want_std;
     c->launches += 1;
     if (timed) cudaEventRecord(c->ev[5][0], c->stream);
@@ -572,6 +539,66 @@ int collect_timing(cutoff_ctx* c) {
 }
 
 bool valid_latent(int D) { return D == 4 || D == 8 || D == 16 || D == 32; }
+
+// Kernels that need more than 48 KB of dynamic shared memory must be told so once per device.  Done at
+// context creation, with the context's device current, for every kernel this context's shape can launch
+// (a function attribute belongs to the device's copy of the kernel, not to the process).
+template <typename Kernel>
+cudaError_t allow_smem(Kernel kernel, size_t bytes) {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+}
+
+template <int E>
+cudaError_t allow_smem_sort() {
+    cudaError_t e = allow_smem(k_sort_sum_tma<E, false>, 100 * 1024);
+    if (e == cudaSuccess) e = allow_smem(k_sort_sum_tma<E, true>, 100 * 1024);
+    return e;
+}
+
+template <int D>
+cudaError_t allow_smem_chain() {
+    cudaError_t e = allow_smem(k_chain<D>, 220 * 1024);
+    if (e == cudaSuccess) e = allow_smem(k_chain_resident<D>, 220 * 1024);
+    if (e == cudaSuccess) e = allow_smem(k_chain_literal<D>, 220 * 1024);
+    return e;
+}
+
+cudaError_t set_kernel_attributes(const cutoff_ctx* c) {
+    cudaError_t e = cudaSuccess;
+    switch (c->P) {
+        case 32: e = allow_smem_sort<1>(); break;
+        case 64: e = allow_smem_sort<2>(); break;
+        case 128: e = allow_smem_sort<4>(); break;
+        case 256: e = allow_smem_sort<8>(); break;
+        case 512: e = allow_smem_sort<16>(); break;
+        case 1024: e = allow_smem_sort<32>(); break;
+        default: break;
+    }
+    if (e != cudaSuccess) return e;
+    switch (c->D) {
+        case 4: e = allow_smem_chain<4>(); break;
+        case 8: e = allow_smem_chain<8>(); break;
+        case 16: e = allow_smem_chain<16>(); break;
+        default: e = allow_smem_chain<32>(); break;
+    }
+    if (e != cudaSuccess) return e;
+    switch (c->H) {
+        case 32: e = allow_smem(k_enc_rnn_resident<8>, 200 * 1024); break;
+        case 64: e = allow_smem(k_enc_rnn_resident<16>, 200 * 1024); break;
+        case 128: e = allow_smem(k_enc_rnn_resident<32>, 200 * 1024); break;
+        case 256: e = allow_smem(k_enc_rnn_resident<64>, 200 * 1024); break;
+        default: break;
+    }
+    if (e == cudaSuccess) e = allow_smem(k_enc_rnn_cluster, 200 * 1024);
+    if (e != cudaSuccess || !c->use_tc) return e;
+    e = allow_smem(tc::k_emit_tc, tc::kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(tc::k_gemm_relu_tc, tc::kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(tc::k_emit_dual_tc, tc::kDualSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc_literal, 227 * 1024);
+    return e;
+}
 
 }  // namespace
 
@@ -626,7 +653,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
         if (err__ != cudaSuccess) return fail(err__ == cudaErrorMemoryAllocation ? CUTOFF_ERR_NOMEM : CUTOFF_ERR_CUDA); \
     } while (0)
 
-    CREATE_CHECK(cudaSetDevice(cfg->device));
+    DeviceGuard guard(cfg->device);
+    CREATE_CHECK(guard.err);
     if ((cfg->flags & CUTOFF_FLAG_GRAPH) && !c->stream) {
         // the default stream cannot be captured: graph mode without a caller stream runs on its own
         CREATE_CHECK(cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking));
@@ -698,6 +726,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
             rc = make_tile_map(c, &c->map_r, c->d_r, static_cast<uint64_t>(c->alloc_rows), static_cast<uint64_t>(c->H));
         if (rc) return fail(rc);
     }
+    CREATE_CHECK(set_kernel_attributes(c));
     CREATE_CHECK(cudaMallocHost(&c->h_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMallocHost(&c->h_state, sizeof(DevState)));
     CREATE_CHECK(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
@@ -710,7 +739,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
 
 void cutoff_destroy(cutoff_ctx* ctx) {
     if (!ctx) return;
-    cudaSetDevice(ctx->cfg.device);
+    DeviceGuard guard(ctx->cfg.device);
     cudaStreamSynchronize(ctx->stream);
     free_all(ctx);
     delete ctx;
@@ -733,7 +762,8 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     for (size_t i = 0; i < total; ++i)
         if (!std::isfinite(src[i])) return CUTOFF_ERR_BAD_BLOB;
 
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     // device layout: every tensor starts on a 32-byte boundary (16-byte loads and tensor maps need aligned bases)
     std::vector<size_t> off(specs.size());
@@ -991,7 +1021,8 @@ static int push_common(cutoff_ctx* c, const float* dev_src) {
 
 int cutoff_push_async(cutoff_ctx* c, const float* runtimes_sec_device) {
     if (!c || !runtimes_sec_device) return CUTOFF_ERR_BAD_ARG;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     return push_common(c, runtimes_sec_device);
 }
 
@@ -1027,7 +1058,7 @@ static int push_censored(cutoff_ctx* c, const float* runtimes_sec, int on_device
     if (rc) return rc;
     CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
-    if (c->h_state->error_flags & kErrBadValue) {
+    if (c->h_state->error_flags & (kErrBadValue | kErrNoFinisher)) {
         c->pushes = c->h_state->push_count;
         CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
         return CUTOFF_ERR_BAD_VALUE;
@@ -1037,7 +1068,8 @@ static int push_censored(cutoff_ctx* c, const float* runtimes_sec, int on_device
 
 int cutoff_push(cutoff_ctx* c, const float* runtimes_sec, int on_device, const uint8_t* censored) {
     if (!c || !runtimes_sec) return CUTOFF_ERR_BAD_ARG;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     if (censored) return push_censored(c, runtimes_sec, on_device, censored);
     if (!on_device) {
         for (int j = 0; j < c->N; ++j)
@@ -1063,8 +1095,9 @@ int cutoff_push(cutoff_ctx* c, const float* runtimes_sec, int on_device, const u
 int cutoff_predict_async(cutoff_ctx* c) {
     if (!c) return CUTOFF_ERR_BAD_ARG;
     if (!c->weights_loaded) return CUTOFF_ERR_STATE;
-    if (c->pending) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    if (c->pending || c->partial_pending) return CUTOFF_ERR_STATE;
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     c->pending = true;
     c->pending_warmup = c->pushes < static_cast<uint32_t>(c->W);
     if (c->pending_warmup) {
@@ -1080,7 +1113,8 @@ int cutoff_predict_async(cutoff_ctx* c) {
 int cutoff_fetch(cutoff_ctx* c, int32_t* c_out) {
     if (!c || !c_out) return CUTOFF_ERR_BAD_ARG;
     if (!c->pending) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     c->pending = false;
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     if (c->h_state->error_flags & kErrBadValue) {
@@ -1156,7 +1190,8 @@ int cutoff_step(cutoff_ctx* c, const float* runtimes_sec, int32_t* c_out) {
     }
     for (int j = 0; j < c->N; ++j)
         if (!(runtimes_sec[j] > 0.0f) || !std::isfinite(runtimes_sec[j])) return CUTOFF_ERR_BAD_VALUE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     if (!c->graph_exec) {
         CU_CHECK(c, cudaStreamSynchronize(c->stream));
         const int rc = build_graph(c, true);
@@ -1185,7 +1220,8 @@ int cutoff_step_device(cutoff_ctx* c, const float* runtimes_sec_device, int32_t*
         if (rc < 0) return rc;
         return cutoff_predict(c, c_out);
     }
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     if (!c->graph_dev_exec) {
         CU_CHECK(c, cudaStreamSynchronize(c->stream));
         const int rc = build_graph(c, false);
@@ -1217,7 +1253,8 @@ int cutoff_step_device(cutoff_ctx* c, const float* runtimes_sec_device, int32_t*
 int cutoff_get_stats(cutoff_ctx* c, float* e_out, float* omega_out) {
     if (!c) return CUTOFF_ERR_BAD_ARG;
     if (!c->have_result) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     if (e_out) CU_CHECK(c, cudaMemcpyAsync(e_out, c->d_E, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
     if (omega_out)
         CU_CHECK(c, cudaMemcpyAsync(omega_out, c->d_omega, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
@@ -1228,7 +1265,8 @@ int cutoff_get_stats(cutoff_ctx* c, float* e_out, float* omega_out) {
 int cutoff_get_order_stat_std(cutoff_ctx* c, float* std_sec) {
     if (!c || !std_sec) return CUTOFF_ERR_BAD_ARG;
     if (!c->have_result || !c->have_std) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaMemcpyAsync(std_sec, c->d_std, sizeof(float) * c->N, cudaMemcpyDeviceToHost, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     return CUTOFF_OK;
@@ -1237,7 +1275,8 @@ int cutoff_get_order_stat_std(cutoff_ctx* c, float* std_sec) {
 int cutoff_get_partial_sums(cutoff_ctx* c, double* sums) {
     if (!c || !sums) return CUTOFF_ERR_BAD_ARG;
     if (!c->have_result) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaMemcpyAsync(sums, c->d_sums, sizeof(double) * c->N, cudaMemcpyDeviceToHost, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     return CUTOFF_OK;
@@ -1247,7 +1286,8 @@ int cutoff_decide_from_sums(cutoff_ctx* c, const double* sums, int32_t* c_out) {
     if (!c || !sums || !c_out) return CUTOFF_ERR_BAD_ARG;
     if (c->pending) return CUTOFF_ERR_STATE;
     if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_ERR_STATE;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaMemcpyAsync(c->d_sums, sums, sizeof(double) * c->N, cudaMemcpyHostToDevice, c->stream));
     const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
     k_decide<<<1, kDecideThreads, 0, c->stream>>>(c->d_sums, c->N, 1.0 / static_cast<double>(total), c->d_state, 0,
@@ -1260,14 +1300,107 @@ int cutoff_decide_from_sums(cutoff_ctx* c, const double* sums, int32_t* c_out) {
     return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
 }
 
+int cutoff_predict_partial_async(cutoff_ctx* c) {
+    if (!c) return CUTOFF_ERR_BAD_ARG;
+    if (!c->weights_loaded) return CUTOFF_ERR_STATE;
+    if (c->pending || c->partial_pending) return CUTOFF_ERR_STATE;
+    if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
+    const int rc = enqueue_decision(c, false);
+    if (rc == CUTOFF_OK) c->partial_pending = true;
+    return rc;
+}
+
+int cutoff_partial_sums_device(cutoff_ctx* c, double** sums_device) {
+    if (!c || !sums_device) return CUTOFF_ERR_BAD_ARG;
+    *sums_device = c->d_sums;
+    return CUTOFF_OK;
+}
+
+int cutoff_decide_from_device_sums(cutoff_ctx* c, const double* sums_device, int32_t* c_out) {
+    if (!c || !sums_device || !c_out) return CUTOFF_ERR_BAD_ARG;
+    if (c->pending) return CUTOFF_ERR_STATE;
+    if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_ERR_STATE;
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
+    if (sums_device != c->d_sums)
+        CU_CHECK(c, cudaMemcpyAsync(c->d_sums, sums_device, sizeof(double) * c->N, cudaMemcpyDeviceToDevice, c->stream));
+    const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
+    // the decision counter moves on here if the sums came from cutoff_predict_partial_async (which left it alone)
+    k_decide<<<1, kDecideThreads, 0, c->stream>>>(c->d_sums, c->N, 1.0 / static_cast<double>(total), c->d_state,
+                                                  c->partial_pending ? 1 : 0, c->d_E, c->d_omega);
+    c->launches += 1;
+    CU_CHECK(c, cudaMemcpyAsync(c->h_state, c->d_state, sizeof(DevState), cudaMemcpyDeviceToHost, c->stream));
+    CU_CHECK(c, cudaStreamSynchronize(c->stream));
+    if (c->h_state->error_flags & kErrBadValue) {
+        // a bad asynchronous push came before this decision: as cutoff_fetch reports it
+        c->pushes = c->h_state->push_count;
+        CU_CHECK(c, cudaMemsetAsync(&c->d_state->error_flags, 0, sizeof(int32_t), c->stream));
+        c->partial_pending = false;
+        return CUTOFF_ERR_BAD_VALUE;
+    }
+    if (c->h_state->error_flags & kErrTimeout) return CUTOFF_ERR_TIMEOUT;
+    if (c->partial_pending) {
+        const int rc = collect_timing(c);
+        if (rc) return rc;
+        c->partial_pending = false;
+        c->decided_once = true;
+    }
+    c->have_result = true;
+    *c_out = c->h_state->c_star;
+    return c->h_state->code == 2 ? CUTOFF_DEGENERATE : CUTOFF_OK;
+}
+
+int cutoff_measure_pipe_rates(int device, float* rates_out) {
+    if (device < 0 || !rates_out) return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    cudaDeviceProp prop;
+    CU_CHECK(none, cudaGetDeviceProperties(&prop, device));
+    const int sms = prop.multiProcessorCount;
+    long long* d_cycles = nullptr;
+    float* d_sink = nullptr;
+    if (cudaMalloc(&d_cycles, sizeof(long long) * sms) != cudaSuccess || cudaMalloc(&d_sink, sizeof(float)) != cudaSuccess) {
+        cudaFree(d_cycles);
+        return CUTOFF_ERR_NOMEM;
+    }
+    std::vector<long long> h(sms);
+    int rc = CUTOFF_OK;
+    for (int kind = 0; kind < 3 && rc == CUTOFF_OK; ++kind) {
+        double best = 0.0;
+        for (int rep = 0; rep < 4 && rc == CUTOFF_OK; ++rep) {         // the first repetition warms the clocks up
+            if (kind == 0) k_pipe_rate<0><<<sms, kRateThreads>>>(1.25f, d_cycles, d_sink);
+            if (kind == 1) k_pipe_rate<1><<<sms, kRateThreads>>>(1.25f, d_cycles, d_sink);
+            if (kind == 2) k_pipe_rate<2><<<sms, kRateThreads>>>(1.25f, d_cycles, d_sink);
+            if (cudaMemcpy(h.data(), d_cycles, sizeof(long long) * sms, cudaMemcpyDeviceToHost) != cudaSuccess) {
+                rc = CUTOFF_ERR_CUDA;
+                break;
+            }
+            long long worst = 1;
+            for (long long v : h) worst = v > worst ? v : worst;
+            const double warp_instr = static_cast<double>(kRateThreads / 32) * kRateChains * kRateIters;
+            const double rate = warp_instr / static_cast<double>(worst);
+            if (rep > 0 && rate > best) best = rate;
+        }
+        rates_out[kind] = static_cast<float>(best);
+    }
+    cudaFree(d_cycles);
+    cudaFree(d_sink);
+    return rc;
+}
+
 int cutoff_reset(cutoff_ctx* c) {
     if (!c) return CUTOFF_ERR_BAD_ARG;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
     CU_CHECK(c, cudaMemsetAsync(c->d_ring, 0, sizeof(float) * c->W * c->N, c->stream));
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     c->pushes = 0;
     c->pending = false;
+    c->partial_pending = false;
     c->have_result = false;
     c->draws_valid = false;
     c->proj_stale = true;
@@ -1279,7 +1412,8 @@ int cutoff_save_state(cutoff_ctx* c, void* buf, size_t* nbytes) {
     const size_t need = 4 * sizeof(uint32_t) + sizeof(DevState) + sizeof(float) * c->W * c->N;
     if (!buf) { *nbytes = need; return CUTOFF_OK; }
     if (*nbytes < need) return CUTOFF_ERR_BAD_ARG;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     char* p = static_cast<char*>(buf);
     const uint32_t hdr[4] = {0x53465443u /* "CTFS" */, 1u, static_cast<uint32_t>(c->N), static_cast<uint32_t>(c->W)};
     std::memcpy(p, hdr, sizeof(hdr));
@@ -1303,14 +1437,17 @@ int cutoff_restore_state(cutoff_ctx* c, const void* buf, size_t nbytes) {
         return CUTOFF_ERR_BAD_ARG;
     DevState s;
     std::memcpy(&s, p + sizeof(hdr), sizeof(s));
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     CU_CHECK(c, cudaMemcpy(c->d_state, &s, sizeof(DevState), cudaMemcpyHostToDevice));
     CU_CHECK(c, cudaMemcpy(c->d_ring, p + sizeof(hdr) + sizeof(DevState), sizeof(float) * c->W * c->N,
                            cudaMemcpyHostToDevice));
     c->pushes = s.push_count;
     c->pending = false;
+    c->partial_pending = false;
     c->have_result = false;
+    c->draws_valid = false;            // the retained draws belong to a decision on the state that was replaced
     c->proj_stale = true;
     return CUTOFF_OK;
 }
@@ -1341,8 +1478,10 @@ int cutoff_set_option(cutoff_ctx* c, const char* name, int64_t value) {
         return CUTOFF_OK;
     }
     if (std::strcmp(name, "pass_rows") == 0) {
-        if (value < 1024) return CUTOFF_ERR_BAD_ARG;
+        if (value < 1024 || value > 0x7fffffffll) return CUTOFF_ERR_BAD_ARG;
+        if (c->graph_exec || c->graph_dev_exec) return CUTOFF_ERR_STATE;   // the captured graph replays the old split
         plan_chunks(c, static_cast<int>(value));
+        c->draws_valid = false;
         return CUTOFF_OK;
     }
     return CUTOFF_ERR_BAD_ARG;
@@ -1378,7 +1517,8 @@ int cutoff_debug_normals(int device, uint64_t seed, uint32_t step, uint32_t stre
     if (device < 0 || k0 < 0 || count < 1 || n_elems < 1 || k0 + count > (1ll << 32)) return CUTOFF_ERR_BAD_ARG;
     if (!normals_out && !words_out) return CUTOFF_ERR_BAD_ARG;
     cutoff_ctx* none = nullptr;
-    CU_CHECK(none, cudaSetDevice(device));
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
     const int nq = (n_elems + 3) / 4;
     float* d_n = nullptr;
     uint32_t* d_w = nullptr;
@@ -1407,7 +1547,8 @@ int cutoff_debug_samples(cutoff_ctx* c, int64_t k0, int64_t count, float* x_out)
     if (!c || !x_out || k0 < 0 || count < 1 || k0 + count > c->S) return CUTOFF_ERR_BAD_ARG;
     if (!c->weights_loaded || c->pending) return CUTOFF_ERR_STATE;
     if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     c->draws_valid = false;                                 // the sample matrix is about to be overwritten
     launch_encoder(c);
     for (int64_t done = 0; done < count; done += c->chunk_rows) {
@@ -1427,7 +1568,8 @@ int cutoff_debug_window(cutoff_ctx* c, float* window_out) {
     if (!c || !window_out) return CUTOFF_ERR_BAD_ARG;
     if (c->pending) return CUTOFF_ERR_STATE;
     if (c->pushes < static_cast<uint32_t>(c->W)) return CUTOFF_WARMUP;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     CU_CHECK(c, cudaStreamSynchronize(c->stream));
     for (int t = 0; t < c->W; ++t) {                       // position t (0 = oldest) sits in slot (pushes + t) mod W
         const size_t slot = (static_cast<size_t>(c->pushes) + t) % c->W;
@@ -1440,7 +1582,8 @@ int cutoff_debug_window(cutoff_ctx* c, float* window_out) {
 int cutoff_debug_sort(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t n, float* keys_out, int32_t* perm_out) {
     if (!c || !rows || !keys_out || !perm_out || n_rows < 1 || n < 1 || n > 4096 || n_rows > (1 << 24))
         return CUTOFF_ERR_BAD_ARG;
-    CU_CHECK(c, cudaSetDevice(c->cfg.device));
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
     const size_t elems = static_cast<size_t>(n_rows) * n;
     float *d_rows = nullptr, *d_keys = nullptr;
     int* d_perm = nullptr;
@@ -1476,12 +1619,48 @@ int cutoff_debug_sort(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t 
     return rc;
 }
 
+int cutoff_debug_sort_values(cutoff_ctx* c, const float* rows, int64_t n_rows, int32_t n, float* keys_out) {
+    if (!c || !rows || !keys_out || n_rows < 1 || n < 1 || n > 4096 || n_rows > (1 << 24)) return CUTOFF_ERR_BAD_ARG;
+    DeviceGuard guard(c->cfg.device);
+    CU_CHECK(c, guard.err);
+    const size_t elems = static_cast<size_t>(n_rows) * n;
+    float *d_rows = nullptr, *d_keys = nullptr;
+    int rc = CUTOFF_OK;
+    if (cudaMalloc(&d_rows, elems * 4) != cudaSuccess || cudaMalloc(&d_keys, elems * 4) != cudaSuccess) rc = CUTOFF_ERR_NOMEM;
+    if (!rc && cudaMemcpyAsync(d_rows, rows, elems * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess) rc = CUTOFF_ERR_CUDA;
+    if (!rc) {
+        const int P = next_pow2(n) < 32 ? 32 : next_pow2(n);
+        const int rows_i = static_cast<int>(n_rows);
+        const int grid_w = ceil_div(rows_i, kSortWarps) < 4 * c->sm_count ? ceil_div(rows_i, kSortWarps) : 4 * c->sm_count;
+        const int grid_c = rows_i < 4 * c->sm_count ? rows_i : 4 * c->sm_count;
+        switch (P) {
+            case 32: k_debug_sort_values_warp<1><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 64: k_debug_sort_values_warp<2><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 128: k_debug_sort_values_warp<4><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 256: k_debug_sort_values_warp<8><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 512: k_debug_sort_values_warp<16><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 1024: k_debug_sort_values_warp<32><<<grid_w, kSortWarps * 32, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            case 2048: k_debug_sort_values_cta<2><<<grid_c, 64, 0, c->stream>>>(d_rows, n, rows_i, d_keys); break;
+            default: k_debug_sort_values_cta<4><<<grid_c, 128, 0, c->stream>>>(d_rows, n, rows_i, d_keys);
+        }
+        c->launches += 1;
+        if (cudaMemcpyAsync(keys_out, d_keys, elems * 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess ||
+            cudaStreamSynchronize(c->stream) != cudaSuccess)
+            rc = CUTOFF_ERR_CUDA;
+    }
+    if (rc == CUTOFF_ERR_CUDA) c->last_error = cudaGetErrorString(cudaGetLastError());
+    cudaFree(d_rows); cudaFree(d_keys);
+    return rc;
+}
+
 }  // extern "C"
 
 // ---- allocation-free entry point -------------------------------------------------------------
 
 namespace {
 constexpr int kStaticParts = 256;     // partial rows (= most CTAs the sort kernel may use here)
+constexpr int kStaticRowsPerWarp = 64;                                                  // rows a warp adds in fp32
+constexpr int64_t kStaticBlockRows = static_cast<int64_t>(kStaticParts) * kSortWarps * kStaticRowsPerWarp;   // 131072
 static_assert(kStaticParts * CUTOFF_STATIC_MAX_N * sizeof(float) == CUTOFF_STATIC_SCRATCH_BYTES, "scratch size");
 
 // Scratch of cutoff_sorted_row_sums_static: one partial sum row per CTA.  Lives in the library
@@ -1500,10 +1679,12 @@ void launch_static_sort(const float* x, int ldx, int n, int n_rows, int grid, fl
 
 extern "C" int cutoff_sorted_row_sums_static(int device, const float* x, int64_t n_rows, int32_t n, int32_t ldx,
                                              double* sums, void* stream) {
-    if (device < 0 || device >= kMaxDevices || !x || !sums || n_rows < 1 || n_rows > 0x7fffffffll || n < 1 || ldx < n)
+    if (device < 0 || device >= kMaxDevices || !x || !sums || n_rows < 1 || n_rows > CUTOFF_STATIC_MAX_ROWS || n < 1 ||
+        ldx < n)
         return CUTOFF_ERR_BAD_ARG;
     if (n > CUTOFF_STATIC_MAX_N) return CUTOFF_ERR_TOO_LARGE;
-    if (cudaSetDevice(device) != cudaSuccess) return CUTOFF_ERR_CUDA;
+    DeviceGuard guard(device);
+    if (guard.err != cudaSuccess) return CUTOFF_ERR_CUDA;
     if (!g_static_partial_addr[device]) {
         // once per device, with that device current: translate the symbol into a device address
         float* addr = nullptr;
@@ -1513,20 +1694,26 @@ extern "C" int cutoff_sorted_row_sums_static(int device, const float* x, int64_t
     }
     float* partial = g_static_partial_addr[device];
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int rows = static_cast<int>(n_rows);
-    const int want = ceil_div(rows, kSortWarps);
-    const int grid = want < kStaticParts ? want : kStaticParts;
     const int P = next_pow2(n) < 32 ? 32 : next_pow2(n);
-    // every CTA of the grid writes its whole partial row (zeros if it had no sample), and the
-    // column sum reads exactly `grid` rows: stale contents of the shared array are never read
-    switch (P) {
-        case 32: launch_static_sort<1>(x, ldx, n, rows, grid, partial, s); break;
-        case 64: launch_static_sort<2>(x, ldx, n, rows, grid, partial, s); break;
-        case 128: launch_static_sort<4>(x, ldx, n, rows, grid, partial, s); break;
-        case 256: launch_static_sort<8>(x, ldx, n, rows, grid, partial, s); break;
-        case 512: launch_static_sort<16>(x, ldx, n, rows, grid, partial, s); break;
-        default: launch_static_sort<32>(x, ldx, n, rows, grid, partial, s); break;
+    // The rows go through in blocks of kStaticBlockRows: within a block a warp adds at most kStaticRowsPerWarp
+    // sorted rows in fp32, then the block's partial rows are added to `sums` in double.  The blocks run one after
+    // the other on the stream, so they can share the scratch array.
+    for (int64_t r0 = 0; r0 < n_rows; r0 += kStaticBlockRows) {
+        const int rows = static_cast<int>(n_rows - r0 < kStaticBlockRows ? n_rows - r0 : kStaticBlockRows);
+        const int want = ceil_div(rows, kSortWarps);
+        const int grid = want < kStaticParts ? want : kStaticParts;
+        const float* xb = x + static_cast<size_t>(r0) * ldx;
+        // every CTA of the grid writes its whole partial row (zeros if it had no sample), and the
+        // column sum reads exactly `grid` rows: stale contents of the shared array are never read
+        switch (P) {
+            case 32: launch_static_sort<1>(xb, ldx, n, rows, grid, partial, s); break;
+            case 64: launch_static_sort<2>(xb, ldx, n, rows, grid, partial, s); break;
+            case 128: launch_static_sort<4>(xb, ldx, n, rows, grid, partial, s); break;
+            case 256: launch_static_sort<8>(xb, ldx, n, rows, grid, partial, s); break;
+            case 512: launch_static_sort<16>(xb, ldx, n, rows, grid, partial, s); break;
+            default: launch_static_sort<32>(xb, ldx, n, rows, grid, partial, s); break;
+        }
+        k_colsum<<<ceil_div(n, 256), 256, 0, s>>>(partial, grid, n, sums, r0 > 0 ? 1 : 0);
     }
-    k_colsum<<<ceil_div(n, 256), 256, 0, s>>>(partial, grid, n, sums);
     return cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
 }

@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(kPushThreads) k_push(const float* __restrict__
         if (!(v > 0.0f) || !isfinite(v)) bad = 1;
         s += static_cast<double>(v);
     }
+    if (tid == 0 && (st->error_flags & kErrNoFinisher)) bad = 1;   // raised by the imputation that precedes this push
     bad = __syncthreads_or(bad);
     if (bad) {
         if (tid == 0) st->error_flags |= kErrBadValue;
@@ -65,7 +66,7 @@ constexpr uint32_t kStreamImpute = 0x300u;
 
 __global__ void __launch_bounds__(kImputeThreads) k_impute(float* __restrict__ stage, const uint8_t* __restrict__ censored,
                                                             const float* __restrict__ x, int ldx, int S, int N,
-                                                            const DevState* __restrict__ st, NoiseKey key) {
+                                                            DevState* __restrict__ st, NoiseKey key) {
     __shared__ float red[kImputeThreads / 32];
     __shared__ float s_threshold;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -83,7 +84,13 @@ __global__ void __launch_bounds__(kImputeThreads) k_impute(float* __restrict__ s
         if (lane == 0) s_threshold = m;
     }
     __syncthreads();
-    const float threshold = s_threshold;          // -inf if nobody finished: the push that follows rejects the vector
+    const float threshold = s_threshold;
+    if (!(threshold > -INFINITY)) {
+        // nobody finished, so there is no cutoff time to truncate at: flag the vector; the push kernel that
+        // follows sees the flag and leaves the window untouched
+        if (threadIdx.x == 0) st->error_flags |= kErrNoFinisher;
+        return;
+    }
     const float scale = st->scale;
     const uint32_t step = st->step;
     for (int j = warp; j < N; j += kImputeThreads / 32) {

@@ -474,7 +474,8 @@ __global__ void __launch_bounds__(kDecideThreads) k_decide(const double* __restr
 
 // ---------------------------------------------------------------------------------------------
 // Column sums of the partial rows, in a fixed order, in double, followed by the decision in the
-// CTA that finishes last (a ticket counter in the device state; nobody waits on anybody).
+// CTA that finishes last (a ticket counter in the device state; nobody waits on anybody); decide = 0
+// stops after the sums.
 // A CTA covers 32 columns with 32 row slices; slice s adds rows s, s+32, ...; the slices are then
 // added in order.
 // ---------------------------------------------------------------------------------------------
@@ -485,7 +486,7 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
                                                                    double* sums, double inv_samples, DevState* st,
                                                                    float* __restrict__ e_out, float* __restrict__ omega_out,
                                                                    const float* __restrict__ partial_sq,
-                                                                   float* __restrict__ std_out) {
+                                                                   float* __restrict__ std_out, int decide) {
     __shared__ double red[kColsumSlices][32];
     __shared__ bool is_last;
     const int col = blockIdx.x * 32 + (threadIdx.x & 31), slice = threadIdx.x >> 5;
@@ -536,6 +537,7 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
         for (int k = 0; k < kColsumSlices; ++k) total += red[k][threadIdx.x];
         sums[col] = total;
     }
+    if (!decide) return;                                // only the sums were asked for
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -550,12 +552,13 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
     }
 }
 
-// Plain column sums of partial rows (fixed order, double): one thread per column.
+// Plain column sums of partial rows (fixed order, double): one thread per column.  With `accumulate` the
+// result is added to what sums already holds.
 __global__ void __launch_bounds__(256) k_colsum(const float* __restrict__ partial, int n_part, int N,
-                                                double* __restrict__ sums) {
+                                                double* __restrict__ sums, int accumulate) {
     const int j = blockIdx.x * 256 + threadIdx.x;
     if (j >= N) return;
-    double s = 0.0;
+    double s = accumulate ? sums[j] : 0.0;
     for (int p = 0; p < n_part; ++p) s += static_cast<double>(partial[static_cast<size_t>(p) * N + j]);
     sums[j] = s;
 }
@@ -619,6 +622,52 @@ __global__ void __launch_bounds__(WPR * 32) k_debug_sort_cta(const float* __rest
                 keys[static_cast<size_t>(row) * n + idx] = composite_key(v[r]);
                 perm[static_cast<size_t>(row) * n + idx] = static_cast<int>(v[r] & 0xffffffffu);
             }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Test hook: the float instantiation of the networks -- the one the decision path runs -- applied to
+// caller rows, the sorted rows written out instead of summed.  Rows are loaded, padded and sorted
+// exactly as k_sort_sum_* do it.
+// ---------------------------------------------------------------------------------------------
+template <int E>
+__global__ void __launch_bounds__(kSortWarps * 32) k_debug_sort_values_warp(const float* __restrict__ rows, int n, int n_rows,
+                                                                             float* __restrict__ keys) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int row = blockIdx.x * kSortWarps + warp; row < n_rows; row += gridDim.x * kSortWarps) {
+        float v[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int e = r * 32 + lane;
+            v[r] = e < n ? rows[static_cast<size_t>(row) * n + e] : INFINITY;
+        }
+        warp_bitonic_sort<float, E>(v, lane);
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int idx = lane * E + r;
+            if (idx < n) keys[static_cast<size_t>(row) * n + idx] = v[r];
+        }
+    }
+}
+
+template <int WPR>
+__global__ void __launch_bounds__(WPR * 32) k_debug_sort_values_cta(const float* __restrict__ rows, int n, int n_rows,
+                                                                     float* __restrict__ keys) {
+    __shared__ float xch[WPR * 1024];
+    constexpr int E = 32, T_ = WPR * 32;
+    for (int row = blockIdx.x; row < n_rows; row += gridDim.x) {
+        float v[E];
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int e = r * T_ + threadIdx.x;
+            v[r] = e < n ? rows[static_cast<size_t>(row) * n + e] : INFINITY;
+        }
+        cta_bitonic_sort<float, WPR>(v, xch);
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+            const int idx = threadIdx.x * E + r;
+            if (idx < n) keys[static_cast<size_t>(row) * n + idx] = v[r];
         }
     }
 }

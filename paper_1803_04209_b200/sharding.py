@@ -20,23 +20,38 @@ def shard_config(rank: int, world: int, samples_per_rank: int) -> dict:
 
 
 class ShardedDecision:
-    """Wraps a context (anything with predict / get_partial_sums / decide_from_sums) and a process group."""
+    """Wraps a context and a process group.
+
+    With ``device="cuda"`` the context must be a library context whose stream is torch's current stream:
+    its part of the decision is enqueued up to the per-position sums, those N doubles are all-reduced in
+    place in the library's own device array (NCCL orders itself after the work already on the current
+    stream), and the decision is finished from them -- nothing passes through the host.  With
+    ``device=None`` (gloo on CPU) the sums travel through host arrays via get_partial_sums /
+    decide_from_sums.
+    """
 
     def __init__(self, ctx, group=None, device=None):
         self.ctx = ctx
         self.group = group
-        self.device = device           # where the all-reduce buffer lives ("cuda" for NCCL, None/cpu for gloo)
+        self.device = device           # "cuda" for NCCL, None for gloo on CPU
+        self._sums = None
 
     def predict(self):
         """(code, c): the decision over all ranks' samples; identical on every rank."""
         import torch
         import torch.distributed as dist
 
+        if self.device is not None and hasattr(self.ctx, "predict_partial_async"):
+            code = self.ctx.predict_partial_async()
+            if code == 1:              # warm-up: nothing was drawn, nothing to exchange
+                return code, self.ctx.N
+            if self._sums is None:
+                self._sums = self.ctx.partial_sums_tensor()
+            dist.all_reduce(self._sums, op=dist.ReduceOp.SUM, group=self.group)
+            return self.ctx.decide_from_device_sums(self._sums)
         code, c = self.ctx.predict()
-        if code == 1:                  # warm-up: nothing was drawn, nothing to exchange
+        if code == 1:
             return code, c
         sums = torch.from_numpy(np.ascontiguousarray(self.ctx.get_partial_sums()))
-        if self.device is not None:
-            sums = sums.to(self.device)
         dist.all_reduce(sums, op=dist.ReduceOp.SUM, group=self.group)
-        return self.ctx.decide_from_sums(sums.cpu().numpy())
+        return self.ctx.decide_from_sums(sums.numpy())

@@ -109,6 +109,30 @@ def test_sort_permutation_bit_exact(n):
     assert np.array_equal(keys, np.take_along_axis(rows, want_perm, axis=1))
 
 
+@pytest.mark.parametrize("n", [1, 2, 33, 158, 512, 1024, 1025, 2175, 4096])
+def test_float_sort_rows_bit_exact(n):
+    # the fp32 instantiation of the network -- the one every decision runs -- row by row against numpy's sort:
+    # continuous keys, many equal keys, both zeros, infinities among the keys, already sorted and reversed rows
+    rng = np.random.default_rng(1000 + n)
+    rows = [rng.standard_normal(n), rng.lognormal(0.0, 0.5, size=n), rng.integers(-3, 4, size=n) * 0.5,
+            np.full(n, 1.5), np.sort(rng.standard_normal(n)), np.sort(rng.standard_normal(n))[::-1],
+            np.where(rng.random(n) < 0.3, np.inf, rng.standard_normal(n)),
+            np.where(rng.random(n) < 0.5, 0.0, -0.0), rng.standard_normal(n) * 1e-30, rng.standard_normal(n) * 1e30]
+    rows += [rng.standard_normal(n) for _ in range(23)]
+    rows = np.stack(rows).astype(np.float32)
+    gpu = binding.Cutoff(16, 4, 32, 1, 64)
+    got = gpu.debug_sort_values(rows)
+    want = np.sort(rows, axis=1, kind="stable")
+    assert np.array_equal(got, want)                                       # value for value (-0 == +0)
+    nonzero = want != 0
+    assert np.array_equal(got.view(np.uint32)[nonzero], want.view(np.uint32)[nonzero])   # bit for bit
+    assert np.array_equal(np.signbit(got).sum(axis=1), np.signbit(rows).sum(axis=1))     # zeros keep their signs
+    zeros = (got == 0)
+    for r in np.flatnonzero(zeros.any(axis=1)):                            # -0 sorts before +0
+        z = np.signbit(got[r][zeros[r]])
+        assert np.all(z[:-1] >= z[1:])
+
+
 @pytest.mark.parametrize("name,S,offsets", [("tiny", 1024, True), ("tiny", 1024, False), ("n128", 2048, True),
                                             ("n128", 777, False), ("n158", 512, True)])
 def test_sampled_runtimes_fp32(name, S, offsets):
@@ -179,6 +203,13 @@ def test_full_size_sampled_rows_and_invariants(name):
 
 def test_full_size_decision_against_the_full_oracle():
     wl, gpu, orc, prec = make_pair("n1024", steps=inputs.WORKLOADS["n1024"].window + 7)
+    assert_decision_close(gpu, orc.predict(), wl.N)
+
+
+def test_full_size_decision_n4096_against_the_full_oracle():
+    # N = 4096, S = 32768, bf16-representable weights: the whole decision, every sample, against the oracle
+    wl, gpu, orc, prec = make_pair("n4096", steps=inputs.WORKLOADS["n4096"].window + 7)
+    assert gpu.S == 32768
     assert_decision_close(gpu, orc.predict(), wl.N)
 
 
@@ -611,3 +642,92 @@ def test_step_device_equals_step_and_rejects_bad_values():
     a, b, c = host_ctx.step(nxt), dev_ctx.step_device(torch.from_numpy(nxt).cuda()), plain_ctx.step_device(torch.from_numpy(nxt).cuda())
     assert a == b == c
     assert np.array_equal(host_ctx.get_stats()[0], dev_ctx.get_stats()[0])
+
+
+def test_censored_push_refuses_a_mask_without_finishers_and_stale_draws():
+    import torch
+    wl, gpu, orc, prec = make_pair("n128", S=512, steps=inputs.WORKLOADS["n128"].window + 5)
+    observed = inputs.workload_trace(wl, wl.window + 6)[-1]
+    assert gpu.predict()[0] == binding.OK
+    before = gpu.debug_window()
+    # device mask of all ones: nobody finished, so there is no cutoff time to truncate at
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.push(torch.from_numpy(observed).cuda(), torch.ones(wl.N, dtype=torch.uint8, device="cuda"))
+    assert e.value.code == binding.ERR_BAD_VALUE
+    assert np.array_equal(gpu.debug_window(), before)               # the window did not move
+    # the refused push used up this decision's draws: decide again, then save / restore
+    assert gpu.predict()[0] == binding.OK
+    blob = gpu.save_state()
+    gpu.restore_state(blob)
+    censored = np.zeros(wl.N, dtype=bool)
+    censored[:5] = True
+    with pytest.raises(binding.CutoffError) as e:                   # draws of a decision on the replaced state
+        gpu.push(observed, censored)
+    assert e.value.code == binding.ERR_STATE
+    assert gpu.predict()[0] == binding.OK
+    assert gpu.push(observed, censored) == binding.OK
+
+
+def test_pass_rows_cannot_change_under_a_captured_graph():
+    wl = inputs.WORKLOADS["n128"]
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, wl.window + 6)
+    gpu = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, 4096, seed=SEED, flags=binding.FLAG_GRAPH)
+    gpu.load_weights(w)
+    gpu.set_option("pass_rows", 2048)                               # before the capture: fine
+    for x in trace:
+        gpu.step(x)                                                 # the later steps replay the captured graph
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.set_option("pass_rows", 4096)
+    assert e.value.code == binding.ERR_STATE
+    with pytest.raises(binding.CutoffError) as e:
+        gpu.set_option("pass_rows", 1 << 40)
+    assert e.value.code == binding.ERR_BAD_ARG
+    censored = np.zeros(wl.N, dtype=bool)
+    censored[-4:] = True
+    with pytest.raises(binding.CutoffError) as e:                   # two passes: the draws of pass one are gone
+        gpu.push(trace[-1], censored)
+    assert e.value.code == binding.ERR_STATE
+
+
+def test_partial_decisions_add_up_on_the_device():
+    # two contexts draw half of the samples each; their sums are added in the library's own device array and the
+    # decision is finished from there: same result as one context with all samples, nothing through the host
+    import torch
+    S = 2048
+    _, whole, orc, _ = make_pair("n128", S=S, steps=8)
+    _, lo, _, _ = make_pair("n128", S=S // 2, steps=8, sample_offset=0, total_samples=S)
+    _, hi, _, _ = make_pair("n128", S=S // 2, steps=8, sample_offset=S // 2, total_samples=S)
+    code, c = whole.predict()
+    assert lo.predict_partial_async() == binding.OK
+    assert hi.predict_partial_async() == binding.OK
+    with pytest.raises(binding.CutoffError) as e:
+        lo.predict()                                                # a partial decision is open
+    assert e.value.code == binding.ERR_STATE
+    t_lo, t_hi = lo.partial_sums_tensor(), hi.partial_sums_tensor()
+    torch.cuda.synchronize()
+    total = t_lo + t_hi
+    assert np.allclose(total.cpu().numpy(), whole.get_partial_sums(), rtol=1e-6)
+    t_lo.copy_(total)                                               # what an in-place all-reduce leaves behind
+    torch.cuda.synchronize()
+    assert lo.decide_from_device_sums(t_lo) == (code, c)
+    assert hi.decide_from_device_sums(total) == (code, c)
+    assert np.max(np.abs(lo.get_stats()[0] - whole.get_stats()[0]) / whole.get_stats()[0][-1]) <= 1e-6
+    # both contexts advanced their decision counter exactly once: the next shared decision matches the next whole one
+    code2, c2 = whole.predict()
+    lo.predict_partial_async(); hi.predict_partial_async()
+    torch.cuda.synchronize()
+    total = lo.partial_sums_tensor() + hi.partial_sums_tensor()
+    assert np.allclose(total.cpu().numpy(), whole.get_partial_sums(), rtol=1e-6)
+    assert lo.decide_from_device_sums(total) == (code2, c2)
+    assert hi.decide_from_device_sums(total) == (code2, c2)
+    fresh = binding.Cutoff(128, 8, 128, 2, 64)
+    fresh.load_weights(inputs.workload_weights(inputs.WORKLOADS["n128"]))
+    assert fresh.predict_partial_async() == binding.WARMUP
+
+
+def test_measured_pipe_rates_are_plausible():
+    r = binding.measure_pipe_rates(0)
+    assert 1.0 <= r["minmax"] <= 2.1          # 64 lanes per SM per clock = 2 warp-instructions
+    assert 0.5 <= r["shuffle"] <= 1.1         # 32 lanes per SM per clock
+    assert 2.0 <= r["fma"] <= 4.1             # 128 lanes per SM per clock

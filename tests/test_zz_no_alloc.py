@@ -44,6 +44,7 @@ def test_static_scratch_entry_point_matches_the_allocating_path_twice():
     wl, ctx = _context("n1024", 3000)
     x = ctx.debug_samples(0, 3000)                 # the draws of the coming decision
     got = _static_sums(x, torch)
+    assert np.allclose(got, np.sort(x.astype(np.float64), axis=1).sum(axis=0), rtol=1e-6, atol=0)   # the definition
     assert ctx.predict()[0] == binding.OK
     want = ctx.get_partial_sums()
     assert np.allclose(got, want, rtol=1e-6, atol=0)
@@ -51,6 +52,7 @@ def test_static_scratch_entry_point_matches_the_allocating_path_twice():
     wl2, ctx2 = _context("n158", 70)
     x2 = ctx2.debug_samples(0, 70)
     got2 = _static_sums(x2, torch)
+    assert np.allclose(got2, np.sort(x2.astype(np.float64), axis=1).sum(axis=0), rtol=1e-6, atol=0)
     assert ctx2.predict()[0] == binding.OK
     want2 = ctx2.get_partial_sums()
     assert np.allclose(got2, want2, rtol=1e-6, atol=0)
@@ -60,6 +62,20 @@ def test_static_scratch_entry_point_matches_the_allocating_path_twice():
     got3 = _static_sums(x3, torch)
     ctx.predict()
     assert np.allclose(got3, ctx.get_partial_sums(), rtol=1e-6, atol=0)
+
+
+def test_static_scratch_entry_point_many_rows_go_through_in_blocks():
+    # more rows than one pass over the scratch array takes (131072): the sums continue in double across passes,
+    # so a long input loses no more digits than a short one
+    import torch
+    build.build()
+    rng = np.random.default_rng(5)
+    n, rows = 40, 131072 + 4096 + 3
+    x = rng.lognormal(0.0, 0.4, size=(rows, n)).astype(np.float32)
+    want = np.sort(x.astype(np.float64), axis=1).sum(axis=0)
+    for _ in range(2):
+        got = _static_sums(x, torch)
+        assert np.allclose(got, want, rtol=2e-6, atol=0)
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
@@ -76,3 +92,4 @@ def test_static_scratch_entry_point_rejects_what_does_not_fit():
     assert float(sums.abs().sum()) == 0.0          # nothing was written
     assert lib.cutoff_sorted_row_sums_static(0, None, 4, 8, 8, sums.data_ptr(), None) == binding.ERR_BAD_ARG
     assert lib.cutoff_sorted_row_sums_static(0, x.data_ptr(), 4, 8, 4, sums.data_ptr(), None) == binding.ERR_BAD_ARG
+    assert lib.cutoff_sorted_row_sums_static(0, x.data_ptr(), (1 << 24) + 1, 8, 8, sums.data_ptr(), None) == binding.ERR_BAD_ARG
