@@ -274,6 +274,31 @@ int cutoff_debug_sort(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_
  * included) -> keys_out (host, n_rows*n floats, each row ascending).  n <= 4096. */
 int cutoff_debug_sort_values(cutoff_ctx* ctx, const float* rows, int64_t n_rows, int32_t n, float* keys_out);
 
+/* ---- evaluation of cutoff rules on recorded run-times --------------------------------------------
+ * The quantities of the paper's Fig. 2 (Section 4.1), per SGD step t of a recorded trace of worker run-times:
+ * with x~(t) the observed run-times of the step in ascending order (Section 3: Omega(c) = c / x~_(c)),
+ *   best[t], best_c[t]   the ground-truth maximum max_c Omega(c) and the cutoff that attains it (largest c on a tie)
+ *   all[t]               N / x~_(N): the throughput of waiting for all workers
+ *   achieved[m*T + t]    Omega(c) for the cutoff c = cutoffs[m*T + t] that rule m chose for the step (clipped to 1..N)
+ *   step_time[m*T + t]   x~_(c): how long the step lasts under that cutoff, in seconds
+ *   *static_c            the one cutoff that maximises sum_t c / x~_(c)(t) over the whole trace (a static cutoff,
+ *                        as in Chen et al. 2016, cited in Section 1); NULL = not wanted
+ * trace: device, n_steps x ld floats, row t = the N run-times of step t (all finite, > 0), n <= 4096, ld >= n.
+ * cutoffs: device, n_rules x n_steps int32 (NULL if n_rules = 0).  All outputs are device arrays of n_steps
+ * (best_c int32; best, all float), n_rules*n_steps (achieved, step_time) or one element (static_c).
+ * The call waits for its kernels.  Errors: BAD_ARG, NOMEM, CUDA.
+ *
+ * cutoff_order_baseline: the "order" rule of Fig. 4.  For step t > 0 the expected order statistics of n iid
+ * normal run-times by Elfving's formula (Section 3.1.1, in its standard form
+ * mu + sigma * Phi^-1((j - pi/8) / (n - pi/4 + 1))), with mu and sigma the mean and (population) deviation of
+ * every run-time of steps 0 .. t-1, and cutoffs_out[t] = argmax_c c / E[x~_(c)] over positive expectations (largest
+ * c on a tie, n if none); cutoffs_out[0] = n.  cutoffs_out: device, n_steps int32.  Waits.  Errors as above. */
+int cutoff_eval_trace(int device, const float* trace, int64_t n_steps, int32_t n, int32_t ld, const int32_t* cutoffs,
+                      int32_t n_rules, int32_t* best_c, float* best, float* all, float* achieved, float* step_time,
+                      int32_t* static_c, void* stream);
+int cutoff_order_baseline(int device, const float* trace, int64_t n_steps, int32_t n, int32_t ld, int32_t* cutoffs_out,
+                          void* stream);
+
 /* ---- allocation-free entry point ---------------------------------------------------------------
  * The paper has no counterpart for this call.  It serves programs that may not allocate device
  * memory at the time they need order statistics: a server that handed all of the GPU's memory to

@@ -33,7 +33,7 @@ EXPORTS = (
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
     "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
     "cutoff_debug_sort_values", "cutoff_predict_partial_async", "cutoff_partial_sums_device",
-    "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates",
+    "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates", "cutoff_eval_trace", "cutoff_order_baseline",
     "cutoff_sorted_row_sums_static",
 )
 
@@ -101,6 +101,9 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_partial_sums_device": (C.c_int, [vp, C.POINTER(vp)]),
         "cutoff_decide_from_device_sums": (C.c_int, [vp, vp, i32p]),
         "cutoff_measure_pipe_rates": (C.c_int, [C.c_int, f32p]),
+        "cutoff_eval_trace": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, C.c_int32, vp, vp, vp, vp, vp,
+                                        vp, vp]),
+        "cutoff_order_baseline": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
         "cutoff_sorted_row_sums_static": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -366,6 +369,46 @@ def measure_pipe_rates(device: int = 0) -> dict:
     if rc < 0:
         raise CutoffError(rc, "cutoff_measure_pipe_rates")
     return {"minmax": float(out[0]), "shuffle": float(out[1]), "fma": float(out[2])}
+
+
+def eval_trace(trace, cutoffs=None, want_static: bool = True, stream: int | None = None) -> dict:
+    """Scores of cutoff rules on a recorded trace (torch CUDA fp32 [T, N]); cutoffs: torch CUDA int32 [M, T] or None.
+
+    Returns torch CUDA tensors: best_c [T] int32, best [T], all [T], achieved [M, T], step_time [M, T] and, if asked
+    for, static_c (one int32).  Every number is computed by the library's kernels; this only allocates the outputs.
+    """
+    import torch
+    lib = load_library()
+    T, N = trace.shape
+    dev = trace.device
+    M = 0 if cutoffs is None else cutoffs.shape[0]
+    out = {"best_c": torch.empty(T, dtype=torch.int32, device=dev), "best": torch.empty(T, dtype=torch.float32, device=dev),
+           "all": torch.empty(T, dtype=torch.float32, device=dev),
+           "achieved": torch.empty((M, T), dtype=torch.float32, device=dev),
+           "step_time": torch.empty((M, T), dtype=torch.float32, device=dev)}
+    if want_static:
+        out["static_c"] = torch.zeros(1, dtype=torch.int32, device=dev)
+    rc = lib.cutoff_eval_trace(dev.index or 0, trace.data_ptr(), T, N, trace.stride(0),
+                               cutoffs.data_ptr() if M else None, M, out["best_c"].data_ptr(), out["best"].data_ptr(),
+                               out["all"].data_ptr(), out["achieved"].data_ptr() if M else None,
+                               out["step_time"].data_ptr() if M else None,
+                               out["static_c"].data_ptr() if want_static else None, stream or None)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_eval_trace")
+    return out
+
+
+def order_baseline(trace, stream: int | None = None):
+    """Cutoffs of the "order" rule (Elfving's formula on running moments) for a trace (torch CUDA fp32 [T, N])."""
+    import torch
+    lib = load_library()
+    T, N = trace.shape
+    out = torch.empty(T, dtype=torch.int32, device=trace.device)
+    rc = lib.cutoff_order_baseline(trace.device.index or 0, trace.data_ptr(), T, N, trace.stride(0), out.data_ptr(),
+                                   stream or None)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_order_baseline")
+    return out
 
 
 def sorted_row_sums_static(x, sums, n: int | None = None, stream: int | None = None) -> int:

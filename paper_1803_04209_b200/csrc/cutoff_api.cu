@@ -18,6 +18,7 @@
 #include "gemm_tc.cuh"
 #include "chain_tc_literal.cuh"
 #include "pipe_rates.cuh"
+#include "kernels_eval.cuh"
 
 using namespace cutoff;
 
@@ -1651,6 +1652,72 @@ int cutoff_debug_sort_values(cutoff_ctx* c, const float* rows, int64_t n_rows, i
     if (rc == CUTOFF_ERR_CUDA) c->last_error = cudaGetErrorString(cudaGetLastError());
     cudaFree(d_rows); cudaFree(d_keys);
     return rc;
+}
+
+// ---- evaluation of cutoff rules on recorded run-times ------------------------------------------------------
+
+int cutoff_eval_trace(int device, const float* trace, int64_t n_steps, int32_t n, int32_t ld, const int32_t* cutoffs,
+                      int32_t n_rules, int32_t* best_c, float* best, float* all, float* achieved, float* step_time,
+                      int32_t* static_c, void* stream) {
+    if (device < 0 || !trace || n_steps < 1 || n_steps > (1ll << 31) - 1 || n < 1 || n > 4096 || ld < n || n_rules < 0 ||
+        !best_c || !best || !all || (n_rules > 0 && (!cutoffs || !achieved || !step_time)))
+        return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaDeviceProp prop;
+    CU_CHECK(none, cudaGetDeviceProperties(&prop, device));
+    float* d_sorted = nullptr;         // the sorted rows, kept only when the static cutoff is asked for
+    double* d_total = nullptr;
+    if (static_c) {
+        if (cudaMalloc(&d_sorted, sizeof(float) * static_cast<size_t>(n_steps) * n) != cudaSuccess) return CUTOFF_ERR_NOMEM;
+        if (cudaMalloc(&d_total, sizeof(double)) != cudaSuccess) { cudaFree(d_sorted); return CUTOFF_ERR_NOMEM; }
+    }
+    const int P = next_pow2(n) < 32 ? 32 : next_pow2(n);
+    const int cap = 8 * prop.multiProcessorCount;
+    const int64_t want_w = ceil_div64(n_steps, kSortWarps);
+    const int grid_w = static_cast<int>(want_w < cap ? want_w : cap);
+    const int grid_c = static_cast<int>(n_steps < cap ? n_steps : cap);
+#define EVAL_ARGS trace, n_steps, n, ld, cutoffs, n_rules, best_c, best, all, achieved, step_time, d_sorted
+    switch (P) {
+        case 32: k_eval_trace_warp<1><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 64: k_eval_trace_warp<2><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 128: k_eval_trace_warp<4><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 256: k_eval_trace_warp<8><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 512: k_eval_trace_warp<16><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 1024: k_eval_trace_warp<32><<<grid_w, kSortWarps * 32, 0, s>>>(EVAL_ARGS); break;
+        case 2048: k_eval_trace_cta<2><<<grid_c, 64, 0, s>>>(EVAL_ARGS); break;
+        default: k_eval_trace_cta<4><<<grid_c, 128, 0, s>>>(EVAL_ARGS); break;
+    }
+#undef EVAL_ARGS
+    if (static_c) k_best_static<<<1, kStaticThreads, 0, s>>>(d_sorted, n_steps, n, static_c, d_total);
+    const cudaError_t err = cudaStreamSynchronize(s);
+    cudaFree(d_sorted);
+    cudaFree(d_total);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
+}
+
+int cutoff_order_baseline(int device, const float* trace, int64_t n_steps, int32_t n, int32_t ld, int32_t* cutoffs_out,
+                          void* stream) {
+    if (device < 0 || !trace || n_steps < 1 || n_steps > (1ll << 31) - 1 || n < 1 || ld < n || !cutoffs_out)
+        return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double* d_work = nullptr;          // [T] sums / means, [T] sums of squares / deviations, [n] normal quantiles
+    if (cudaMalloc(&d_work, sizeof(double) * (2 * static_cast<size_t>(n_steps) + n)) != cudaSuccess) return CUTOFF_ERR_NOMEM;
+    double* d1 = d_work;
+    double* d2 = d_work + n_steps;
+    double* dq = d_work + 2 * n_steps;
+    k_step_moments<<<static_cast<unsigned>(n_steps), kMomentThreads, 0, s>>>(trace, n_steps, n, ld, d1, d2);
+    k_running_moments<<<1, 32, 0, s>>>(n_steps, n, d1, d2);
+    k_elfving_quantiles<<<ceil_div(n, 256), 256, 0, s>>>(n, dq);
+    k_order_cutoffs<<<static_cast<unsigned>(ceil_div64(n_steps, 8)), 256, 0, s>>>(n_steps, n, d1, d2, dq, cutoffs_out);
+    const cudaError_t err = cudaStreamSynchronize(s);
+    cudaFree(d_work);
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
 }
 
 }  // extern "C"

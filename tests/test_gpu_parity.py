@@ -155,7 +155,7 @@ def test_wide_models_fp32_arithmetic():
     # the large shapes with every product in fp32: isolates the non-tensor-core kernels
     for name, S in (("n1024", 1536), ("n2175", 300), ("n4096", 300)):
         wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 7, precision=0)
-        assert_samples_close(gpu.debug_samples(0, min(S, 256)), orc.samples(np.arange(min(S, 256))), 2e-5)
+        assert_samples_close(gpu.debug_samples(0, min(S, 256)), orc.samples(np.arange(min(S, 256))), TOL_X[0])
         assert_decision_close(gpu, orc.predict(), wl.N)
 
 
@@ -512,7 +512,7 @@ def test_limits_of_the_supported_shapes(N, D, H, lag, S, prec):
     for x in trace:
         gpu.push(x)
         orc.push(x)
-    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec] if prec else 2e-5)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec])
     assert_decision_close(gpu, orc.predict(), N)
 
 
@@ -555,7 +555,7 @@ def test_random_shapes_both_variants(N, D, H, lag, S, prec, literal):
     for x in trace:
         gpu.push(x)
         orc.push(x)
-    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec] if prec else 2e-5)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[prec])
     assert_decision_close(gpu, orc.predict(), N)
 
 
