@@ -136,6 +136,18 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def pipe_rates(device: int, measure: bool) -> dict:
+    """Warp-instructions per clock per SM of fp32 min/max, shuffles and fp32 FMA: measured by the library's
+    micro-benchmark on this GPU, or the nominal figures (64 / 32 / 128 lanes per SM per clock)."""
+    if measure:
+        from paper_1803_04209_b200 import binding
+        r = binding.measure_pipe_rates(device)
+        r["source"] = "measured (cutoff_measure_pipe_rates, this run)"
+        return r
+    return {"minmax": MINMAX_LANES_PER_SM / 32.0, "shuffle": 1.0, "fma": FP32_LANES_PER_SM / 32.0,
+            "source": "nominal lanes per SM per clock"}
+
+
 def cpu_threads() -> int:
     try:
         from threadpoolctl import threadpool_info
@@ -183,6 +195,79 @@ def run_reference(args, wl, weights, trace):
     print(json.dumps(line))
 
 
+def load_weight_file(path: str) -> dict:
+    """Weights saved as an npz of the blob's tensors (what oracle/fit_elbo.py writes)."""
+    with np.load(path) as z:
+        return {k: np.ascontiguousarray(z[k], dtype=np.float32) for k in z.files if not k.startswith("_")}
+
+
+def run_evaluate(args, wl, weights, literal):
+    """Fig. 2's comparison on the workload's synthetic trace: throughput achieved by each cutoff rule relative to
+    the hindsight-best throughput of every step.  All scoring runs in the library's kernels."""
+    import torch
+    from paper_1803_04209_b200 import binding, build, inputs
+    build.build()
+    torch.cuda.set_device(0)
+    n_hist = max(wl.window + 1, min(wl.history, 64))
+    T = args.evaluate_steps
+    trace = inputs.workload_trace(wl, n_hist + T)
+    dev_all = torch.from_numpy(trace).cuda()
+    dev_eval = dev_all[n_hist:]
+    flags = (binding.FLAG_LITERAL if literal else 0) | binding.FLAG_GRAPH
+
+    def model_cutoffs(censor: bool):
+        ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, wl.S, precision=wl.precision, seed=2024,
+                             flags=flags if not censor else flags & ~binding.FLAG_GRAPH)
+        ctx.load_weights(weights)
+        for x in trace[:n_hist]:
+            ctx.push(x)
+        cs = np.empty(T, dtype=np.int32)
+        for t in range(T):
+            # Algorithm 1: the cutoff of step t is set before its run-times arrive ...
+            code, c = ctx.predict()
+            cs[t] = c
+            x = trace[n_hist + t]
+            if censor:
+                # ... and the workers slower than the c-th are killed: their run-times are never observed (Section 4.2)
+                order = np.argsort(x, kind="stable")
+                mask = np.zeros(wl.N, dtype=bool)
+                mask[order[c:]] = True
+                ctx.push(x, mask if mask.any() else None)
+            else:
+                ctx.push(x)
+        ctx.close()
+        return cs
+
+    static = binding.eval_trace(dev_all[:n_hist], None, want_static=True)
+    static_c = int(static["static_c"].item())                       # chosen on the history, applied to what follows
+    order = binding.order_baseline(dev_all)[n_hist:].cpu().numpy()  # its running moments start with the history
+    rules = {"model": model_cutoffs(False), "model_censored": model_cutoffs(True),
+             "static": np.full(T, static_c, dtype=np.int32), "order": order.astype(np.int32),
+             "wait_for_all": np.full(T, wl.N, dtype=np.int32)}
+    names = list(rules)
+    res = binding.eval_trace(dev_eval, torch.from_numpy(np.stack([rules[n] for n in names])).cuda(), want_static=False)
+    best = res["best"].double()
+    report = {}
+    for m, name in enumerate(names):
+        ach = res["achieved"][m].double()
+        report[name] = {"mean_fraction_of_best": float((ach / best).mean()),
+                        "total_fraction_of_best": float(ach.sum() / best.sum()),
+                        "mean_step_seconds": float(res["step_time"][m].double().mean()),
+                        "mean_cutoff": float(np.mean(rules[name]))}
+    fitted = bool(args.weights)
+    line = {"evaluate": {"workload": wl.name, "variant": args.variant, "N": wl.N, "S": wl.S, "steps": T,
+                         "history_steps": n_hist,
+                         "weights": args.weights if fitted else "seeded random initialisation with hand-set bias offsets",
+                         "note": ("model rows use fitted weights" if fitted else
+                                  "the model rows are a plumbing check only: the weights are not fitted to this trace"),
+                         "hindsight_mean_cutoff": float(res["best_c"].double().mean()),
+                         "static_cutoff": static_c, "rules": report,
+                         "how": "throughput c / x~_(c) of every step under each rule's cutoff, relative to the step's "
+                                "maximum over c (known only in hindsight); scored by cutoff_eval_trace / "
+                                "cutoff_order_baseline on the device-resident trace"}}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -201,6 +286,16 @@ def main():
     ap.add_argument("--no-stream", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="launch the kernels of a step one by one instead of replaying the captured graph")
     ap.add_argument("--stream-steps", type=int, default=1000)
+    ap.add_argument("--no-measure-alu-peak", action="store_true",
+                    help="skip the pipe-rate micro-benchmark (a few ms) and take the nominal min/max, shuffle and FMA rates")
+    ap.add_argument("--measure-alu-peak", action="store_true", help="(default) measure those rates in this run")
+    ap.add_argument("--sustained-seconds", type=float, default=2.0,
+                    help="replay the step back to back for this long and report the sustained time per step (0 = skip)")
+    ap.add_argument("--evaluate", action="store_true",
+                    help="score the model's cutoff, a static cutoff, the Elfving 'order' cutoff and waiting for all "
+                         "workers against the hindsight-best throughput on the workload's synthetic trace, then exit")
+    ap.add_argument("--evaluate-steps", type=int, default=200)
+    ap.add_argument("--weights", default="", help="path of a weight file written by oracle/fit_elbo.py (npz); default: seeded random weights")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
         args.warmup = 3
@@ -214,8 +309,13 @@ def main():
     weights = inputs.workload_weights_literal(wl) if literal else inputs.workload_weights(wl)
     trace = inputs.workload_trace(wl, min(wl.history, 64) + args.steps + args.warmup + 8)
 
+    if args.weights:
+        weights = load_weight_file(args.weights)
     if args.impl == "reference":
         run_reference(args, wl, weights, trace)
+        return
+    if args.evaluate:
+        run_evaluate(args, wl, weights, literal)
         return
 
     import torch
@@ -373,7 +473,7 @@ def main():
                           "how": "host clock around cutoff_step (host run-times in, cutoff out), CUDA graph replay"}
         sctx.close()
 
-    # ---- roofline of the dominant stage -----------------------------------------------------------
+    # ---- roofline: the dominant stage, and the path as a whole ------------------------------------------------
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -385,19 +485,23 @@ def main():
     kind, amount = work[dominant]
     dur = stage_avg[dominant] * 1e-3
     smax = peaks.get("sm_max_mhz", 1965.0)
+    # the clock the timed region actually ran at: the median of the nvidia-smi samples taken during it
+    clock_mhz = clocks.get("sm_mhz") or smax
+    rates = pipe_rates(local_rank, measure=not args.no_measure_alu_peak)
+    lane_rate = lambda name: SM_COUNT * 32.0 * rates[name] * clock_mhz * 1e6          # lane-operations per second
+    bf16 = peaks.get("bf16_tflops", 1590.0)
+    tensor_peak = 0.5 * bf16 * 1e12                      # tf32 runs at half the bf16 rate (nominal ratio)
+    tensor_src = ("measured bf16 burst x 0.5 (nominal tf32 : bf16 ratio)" if peaks else "fallback 1590 x 0.5")
     if kind == "tensor":
-        bf16 = peaks.get("bf16_tflops", 1590.0)
-        peak, unit = 0.5 * bf16, "TFLOP/s"             # tf32 runs at half the bf16 rate (nominal ratio)
-        peak_src = ("measured bf16 burst x 0.5 (nominal tf32 : bf16 ratio)" if peaks else "fallback 1590 x 0.5")
-        bound = "tensor"
+        peak, unit, peak_src, bound = tensor_peak / 1e12, "TFLOP/s", tensor_src, "tensor"
     elif dominant == "sort":
-        peak, unit = SM_COUNT * MINMAX_LANES_PER_SM * smax * 1e6 / 1e12, "Tlane-op/s"
-        peak_src = "148 SMs x 64 fp32 min/max lanes x max SM clock"
-        bound = "alu"
+        peak, unit, bound = lane_rate("minmax") / 1e12, "Tlane-op/s", "alu"
+        peak_src = (f"{rates['source']}: {rates['minmax']:.3f} fp32 min/max warp-instructions per clock per SM x 32 lanes "
+                    f"x {SM_COUNT} SMs x {clock_mhz:.0f} MHz (median SM clock sampled during the timed region)")
     else:
-        peak, unit = SM_COUNT * FP32_LANES_PER_SM * smax * 1e6 / 1e12, "Tlane-op/s"
-        peak_src = "148 SMs x 128 fp32 lanes x max SM clock"
-        bound = "alu"
+        peak, unit, bound = lane_rate("fma") / 1e12, "Tlane-op/s", "alu"
+        peak_src = (f"{rates['source']}: {rates['fma']:.3f} fp32 FMA warp-instructions per clock per SM x 32 lanes "
+                    f"x {SM_COUNT} SMs x {clock_mhz:.0f} MHz")
     achieved = amount / dur / 1e12
     traffic = None if literal else NCU_TRAFFIC.get((wl.name, dominant))
     roofline = {"bound": bound, "kernel": dominant, "achieved": achieved, "peak": peak, "unit": unit,
@@ -405,6 +509,63 @@ def main():
                 "traffic_source": traffic["source"] if traffic else None,
                 "algorithmic_per_launch": amount, "peak_source": peak_src,
                 "stage_ms": {k: round(v, 4) for k, v in stage_avg.items()}}
+    # The path's model time: the slowest of the three resources the whole decision needs -- tensor cores (every
+    # product that runs on them), the plain ALUs (the sort's min/max at the measured min/max rate, plus the
+    # multiply-adds of whatever does not run on the tensor cores at the measured FMA rate), and the exchange of keys
+    # between threads (the network's cross-lane stages at the measured shuffle rate).  path_frac sets it against the
+    # measured time of a whole step; frac_vs_nlog2n sets the sort stage against the comparison-sort floor of
+    # N log2 N compare-exchanges per row instead of the network's own count.
+    p2 = 32
+    while p2 < wl.N:
+        p2 *= 2
+    tensor_flops = sum(a for k, (kd, a) in work.items() if kd == "tensor")
+    chain_on_tensor = bool(wl.precision) and wl.D in (16, 32) and not (literal and wl.D == 32)
+    if chain_on_tensor:
+        tensor_flops += 2 * work["chain"][1]
+    fma_ops = sum(a for k, (kd, a) in work.items() if kd == "alu" and k not in ("sort", "chain")) + \
+        (0 if chain_on_tensor else work["chain"][1])
+    minmax_ops = work["sort"][1]
+    e_keys = min(32, p2 // 32)
+    lane_bits = (p2 // e_keys).bit_length() - 1                    # cross-lane (and cross-warp) bits of a key's index
+    xchg_stages = lane_bits * (lane_bits + 1) // 2                 # stages whose partners sit in another thread
+    xchg_ops = wl.S * p2 * xchg_stages                             # one key moved per lane per such stage
+    t_tc = tensor_flops / tensor_peak
+    t_alu = minmax_ops / lane_rate("minmax") + fma_ops / lane_rate("fma")
+    t_xchg = xchg_ops / lane_rate("shuffle")
+    t_model = max(t_tc, t_alu, t_xchg)
+    roofline.update({
+        "path_frac": t_model / (ms_per_step * 1e-3),
+        "path_model_ms": {"tensor": round(t_tc * 1e3, 4), "alu": round(t_alu * 1e3, 4), "exchange": round(t_xchg * 1e3, 4)},
+        "path_model_sources": {
+            "tensor": f"{tensor_flops:.4g} FLOP / ({tensor_src})",
+            "alu": f"{minmax_ops:.4g} min/max + {fma_ops:.4g} multiply-adds (counted from the kernels' source) at the "
+                   f"{rates['source']} min/max and FMA rates, {clock_mhz:.0f} MHz",
+            "exchange": f"{xchg_ops:.4g} keys exchanged between threads ({xchg_stages} cross-thread stages of the network) at the "
+                        f"{rates['source']} shuffle rate"},
+        "frac_vs_nlog2n": (wl.S * p2 * (p2.bit_length() - 1) * 2 / (stage_avg["sort"] * 1e-3)) / lane_rate("minmax"),
+        "pipe_rates": {k: round(rates[k], 4) for k in ("minmax", "shuffle", "fma")},
+        "pipe_rates_source": rates["source"],
+    })
+
+    # ---- sustained: the same step replayed back to back for a few seconds, with the clocks seen -------------
+    sustained = None
+    if args.sustained_seconds > 0 and world == 1:
+        n_rep = max(50, int(args.sustained_seconds / max(ms_per_step * 1e-3, 1e-5)))
+        sampler2 = ClockSampler(local_rank)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        sampler2.start()
+        ev0.record(stream)
+        for i in range(n_rep):
+            step_device((args.warmup + i) % dev_trace.shape[0])
+        ev1.record(stream)
+        ev1.synchronize()
+        clk2 = sampler2.stop()
+        ms_sus = ev0.elapsed_time(ev1) / n_rep
+        sustained = {"steps": n_rep, "ms_per_step": ms_sus, "value": wl.S * wl.N / (ms_sus * 1e-3), "unit": UNIT,
+                     "clocks": clk2, "ms_x_mhz": ms_sus * (clk2.get("sm_mhz") or 0.0),
+                     "how": "the same graph replays back to back, no L2 flush in between (the 268 MB sample matrix "
+                            "alone exceeds the L2), one pair of CUDA events around all of them"}
 
     cpu_baseline = None
     if not args.no_cpu_baseline:
@@ -424,7 +585,7 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_sec * 1e3,
                 "h2d_bytes_per_step": 4 * wl.N, "d2h_bytes_per_step": 40 + 8 * wl.N},
         "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu_baseline,
-        "stream_latency": stream_latency,
+        "stream_latency": stream_latency, "sustained": sustained,
         "timed_region_wall_s": round(wall, 3),
     }
     print(json.dumps(line))
