@@ -6,9 +6,9 @@
 //      out    = B hidden (+ b)        (M=128, N=16 or 32, K=H)
 // is two UMMA groups.  The first writes the hidden pre-activations to TMEM columns [0, H); the
 // epilogue warps read them 64 hidden units ("chunk") at a time, apply bias and activation, round
-// to tf32 and store the chunk as a K-major, 128-byte-swizzled A operand in one of two shared
-// memory buffers; the MMA warp multiplies chunk c with the matching K blocks of B while the
-// epilogue produces chunk c+1.  The second result (mu, or mean | logvar) is read back by all
+// to tf32 and store the chunk as two K-major, 128-byte-swizzled A operand tiles in the buffer of
+// the tile's slot; the MMA warp multiplies that chunk with the matching K blocks of B while the
+// epilogue produces the same chunk of the other tile in flight.  The second result (mu, or mean | logvar) is read back by all
 // epilogue warps, which draw the noise, form the next latent and store it as the next A operand.
 // The last layer's hidden vector v goes to global memory for the emission output GEMM.
 //
@@ -89,7 +89,6 @@ struct ChainSlot {
 __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const int H = a.H, W = a.W;
-    const int n_chunks = H / 32;                                  // a chunk = 32 hidden units = one K block
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (base - raw);
@@ -179,6 +178,13 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     // The second result of a tile (mu: 16 columns, mean | logvar: 32 columns) reuses the first columns of the
     // tile's pre-activation block: those are multiplied only after every warp has read chunk 0.
 
+    // A hidden layer goes to the second GEMM in chunks of 64 units (two K blocks).  Each slot has one chunk buffer
+    // (its two 16 KB tiles); the chunks of the two tiles in flight are produced alternately -- (chunk 0, slot 0),
+    // (chunk 0, slot 1), (chunk 1, slot 0), ... -- so a slot's buffer is being multiplied while the other slot's is
+    // written, and both roles walk the same order.  sl.nu counts a slot's chunks: chunk n completes phase n of
+    // bar_h (written) and of bar_hfree (multiplied).
+    const int n_chunks64 = H / 64;
+
     if (warp == 0) {
         // ---------------- MMA issuer -------------------------------------------------------------------
         const uint32_t idesc_h = instr_desc_tf32(H), idesc_mu = instr_desc_tf32(16), idesc_head = instr_desc_tf32(32);
@@ -208,23 +214,26 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                 const uint32_t b_base = ph < W ? t_wmu : t_w2;
                 const uint32_t slab = ph < W ? 16u * 128u : 32u * 128u;
                 const uint32_t idesc2 = ph < W ? idesc_mu : idesc_head;
+                for (int c = 0; ok && c < n_chunks64; ++c) {        // second GEMM, chunk by chunk as the epilogue delivers
 #pragma unroll
-                for (int s = 0; s < 2; ++s) {                       // second GEMM, chunk by chunk as the epilogue delivers
-                    ChainSlot& sl = slot[s];
-                    if (!ok || sl.tile < 0) continue;
-                    for (int c = 0; c < n_chunks; ++c, ++sl.nu) {
-                        const uint32_t b = sl.nu & 1u;
-                        ok = mbar_wait(sl.bar_h + 8 * b, (sl.nu >> 1) & 1u, abort_flag, a.st);
-                        if (!ok) break;
+                    for (int s = 0; s < 2; ++s) {
+                        ChainSlot& sl = slot[s];
+                        if (!ok || sl.tile < 0) continue;
+                        ok = mbar_wait(sl.bar_h, sl.nu & 1u, abort_flag, a.st);
+                        if (!ok) continue;
+                        ++sl.nu;
                         tc_fence_after();
                         if (lane == 0) {
-                            const uint64_t a_desc = make_smem_desc(sl.t_hb + b * 16384u);
-                            const uint64_t b_desc = make_smem_desc(b_base + c * slab);
 #pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                umma_tf32(sl.tmem, a_desc + 2 * k, b_desc + 2 * k, idesc2, (c | k) != 0 ? 1u : 0u);
-                            umma_commit(sl.bar_hfree + 8 * b);
-                            if (c == n_chunks - 1) umma_commit(sl.bar_acc2);
+                            for (int kb = 0; kb < 2; ++kb) {
+                                const uint64_t a_desc = make_smem_desc(sl.t_hb + kb * 16384u);
+                                const uint64_t b_desc = make_smem_desc(b_base + (2 * c + kb) * slab);
+#pragma unroll
+                                for (int k = 0; k < 4; ++k)
+                                    umma_tf32(sl.tmem, a_desc + 2 * k, b_desc + 2 * k, idesc2, (c | kb | k) != 0 ? 1u : 0u);
+                            }
+                            umma_commit(sl.bar_hfree);
+                            if (c == n_chunks64 - 1) umma_commit(sl.bar_acc2);
                         }
                         __syncwarp();
                     }
@@ -243,6 +252,8 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         const int row = q * 32 + lane;                                            // TMEM lane = sample of the tile
         const uint32_t lane_off = static_cast<uint32_t>(q * 32) << 16;
         const uint32_t step = a.st->step;
+        const uint32_t hb_off = static_cast<uint32_t>(cg >> 1) * 16384u;          // K block of the chunk this warp writes
+        const int hb_chunk = 4 * (cg & 1);                                        // its first 16-byte chunk in a row
         bool ok = true;
         for (int t0 = blockIdx.x; ok && t0 < n_tiles; t0 += 2 * gridDim.x) {
             slot[0].tile = t0;
@@ -261,59 +272,66 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                 const float* bias = ph < W ? sbzs : (ph == W ? sb1 : sb3);
                 const float* lr = slr + (ph < W ? ph : 0) * H;
                 // ---- hidden layer of both tiles: bias, activation, next A operand (or v) -----------------
+                for (int c = 0; ok && c < n_chunks64; ++c) {
 #pragma unroll
-                for (int s = 0; s < 2; ++s) {
-                    ChainSlot& sl = slot[s];
-                    if (!ok || sl.tile < 0) continue;
-                    ok = mbar_wait(sl.bar_p, sl.np & 1u, abort_flag, a.st);
-                    if (!ok) continue;
-                    ++sl.np;
-                    tc_fence_after();
-                    const int k = sl.tile * 128 + row;
-                    for (int c = 0; c < n_chunks; ++c) {
-                        const int col0 = c * 32 + cg * 8;
-                        uint32_t acc[8];
-                        tmem_ld8(sl.tmem + lane_off + col0, acc);
+                    for (int s = 0; s < 2; ++s) {
+                        ChainSlot& sl = slot[s];
+                        if (!ok || sl.tile < 0) continue;
+                        if (c == 0) {
+                            ok = mbar_wait(sl.bar_p, sl.np & 1u, abort_flag, a.st);
+                            if (!ok) continue;
+                            ++sl.np;
+                            tc_fence_after();
+                        }
+                        const int col0 = c * 64 + cg * 16;
+                        uint32_t acc[16];
+                        tmem_ld16(sl.tmem + lane_off + col0, acc);
                         tmem_ld_wait();
-                        const float4 b_lo = *reinterpret_cast<const float4*>(bias + col0);
-                        const float4 b_hi = *reinterpret_cast<const float4*>(bias + col0 + 4);
-                        const float bv[8] = {b_lo.x, b_lo.y, b_lo.z, b_lo.w, b_hi.x, b_hi.y, b_hi.z, b_hi.w};
-                        float h[8];
-                        if (ph < W) {
-                            const float4 l_lo = *reinterpret_cast<const float4*>(lr + col0);
-                            const float4 l_hi = *reinterpret_cast<const float4*>(lr + col0 + 4);
-                            const float lv[8] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
+                        float h[16];
 #pragma unroll
-                            for (int i = 0; i < 8; ++i) {          // tanh, then (tanh + h_left + h_right) / 3
-                                float e, r;
-                                asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
-                                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-                                h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                        for (int g = 0; g < 4; ++g) {
+                            const float4 bq = *reinterpret_cast<const float4*>(bias + col0 + 4 * g);
+                            const float bv[4] = {bq.x, bq.y, bq.z, bq.w};
+                            if (ph < W) {
+                                const float4 lq = *reinterpret_cast<const float4*>(lr + col0 + 4 * g);
+                                const float lv[4] = {lq.x, lq.y, lq.z, lq.w};
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {      // tanh, then (tanh + h_left + h_right) / 3
+                                    float e, r;
+                                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[4 * g + i]), 2.8853900817779268f, bv[i])));
+                                    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+                                    h[4 * g + i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                                }
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) h[4 * g + i] = fmaxf(__uint_as_float(acc[4 * g + i]) + bv[i], 0.0f);
                             }
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 8; ++i) h[i] = fmaxf(__uint_as_float(acc[i]) + bv[i], 0.0f);
                         }
                         if (ph <= W) {
-                            const uint32_t b = sl.nu & 1u;
-                            if (sl.nu >= 2) {                      // the buffer's previous contents must have been multiplied
-                                ok = mbar_wait(sl.bar_hfree + 8 * b, ((sl.nu >> 1) - 1u) & 1u, abort_flag, a.st);
-                                if (!ok) break;
+                            if (sl.nu >= 1) {                      // the buffer's previous contents must have been multiplied
+                                ok = mbar_wait(sl.bar_hfree, (sl.nu - 1u) & 1u, abort_flag, a.st);
+                                if (!ok) continue;
                             }
-                            const uint32_t dst = sl.t_hb + b * 16384u;
-                            st_shared_v4(dst + sw128(row, 2 * cg), tf32_rna(h[0]), tf32_rna(h[1]), tf32_rna(h[2]), tf32_rna(h[3]));
-                            st_shared_v4(dst + sw128(row, 2 * cg + 1), tf32_rna(h[4]), tf32_rna(h[5]), tf32_rna(h[6]), tf32_rna(h[7]));
+                            const uint32_t dst = sl.t_hb + hb_off;
+#pragma unroll
+                            for (int g = 0; g < 4; ++g)
+                                st_shared_v4(dst + sw128(row, hb_chunk + g), tf32_rna(h[4 * g]), tf32_rna(h[4 * g + 1]),
+                                             tf32_rna(h[4 * g + 2]), tf32_rna(h[4 * g + 3]));
                             fence_proxy_async();
                             tc_fence_before();                     // our TMEM reads of this chunk precede the MMAs it unblocks
                             __syncwarp();
-                            if (lane == 0) mbar_arrive(sl.bar_h + 8 * b);
+                            if (lane == 0) mbar_arrive(sl.bar_h);
                             ++sl.nu;
-                        } else if (k < a.count) {
-                            if (a.round_v) {
+                        } else {
+                            const int k = sl.tile * 128 + row;
+                            if (k < a.count) {
+                                if (a.round_v) {
 #pragma unroll
-                                for (int i = 0; i < 8; ++i) h[i] = tf32_rna(h[i]);
+                                    for (int i = 0; i < 16; ++i) h[i] = tf32_rna(h[i]);
+                                }
+                                store8(a.v_out + static_cast<size_t>(k) * H + col0, h);          // whole 32-byte sectors
+                                store8(a.v_out + static_cast<size_t>(k) * H + col0 + 8, h + 8);
                             }
-                            store8(a.v_out + static_cast<size_t>(k) * H + col0, h);          // one whole 32-byte sector
                         }
                     }
                 }
@@ -323,11 +341,14 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                 for (int s = 0; s < 2; ++s) {
                     ChainSlot& sl = slot[s];
                     if (!ok || sl.tile < 0) continue;
+                    const uint32_t sample = a.sample_base + static_cast<uint32_t>(sl.tile * 128 + row);
+                    float eps[4];                                   // drawn before the wait: the noise does not depend on the result
+                    normal4_fast(static_cast<uint32_t>(cg), sample, ph < W ? static_cast<uint32_t>(ph) : kStreamTransition, step,
+                                 a.key.seed_lo, a.key.seed_hi, eps);
                     ok = mbar_wait(sl.bar_acc2, sl.na & 1u, abort_flag, a.st);
                     if (!ok) continue;
                     ++sl.na;
                     tc_fence_after();
-                    const uint32_t sample = a.sample_base + static_cast<uint32_t>(sl.tile * 128 + row);
                     float z_own[4];
                     if (ph < W) {
                         uint32_t mu_bits[16];
@@ -336,8 +357,6 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                         float mu[16];
 #pragma unroll
                         for (int d = 0; d < 16; ++d) mu[d] = __uint_as_float(mu_bits[d]) + sbmu[d];
-                        float eps[4];
-                        normal4_fast(static_cast<uint32_t>(cg), sample, static_cast<uint32_t>(ph), step, a.key.seed_lo, a.key.seed_hi, eps);
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             const float* wrow = sWsig + (4 * cg + c) * 16;
@@ -355,8 +374,6 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                         tmem_ld16(sl.tmem + lane_off, mean_bits);
                         tmem_ld16(sl.tmem + lane_off + 16, lv_bits);
                         tmem_ld_wait();
-                        float eps[4];
-                        normal4_fast(static_cast<uint32_t>(cg), sample, kStreamTransition, step, a.key.seed_lo, a.key.seed_hi, eps);
 #pragma unroll
                         for (int c = 0; c < 4; ++c) {
                             float mean = 0.0f, lv = 0.0f;
