@@ -100,10 +100,10 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u;
     const uint32_t t_act = base + image_bytes;                    // Z0, Z1, then 4 hidden-chunk buffers: 6 x 16 KB
     // fp32 side tables
-    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz * 2 log2(e)
+    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz
     float* sb1 = sbzs + H;
     float* sb3 = sb1 + H;
-    float* slr = sb3 + H;                    // [W][H]  (h_left + h_right + 1) / 3
+    float* slr = sb3 + H;                    // [W][H]  (h_left + h_right) / 3
     float* sWsig = slr + W * H;              // [16][16]
     float* sbmu = sWsig + 256;
     float* sbsig = sbmu + 16;
@@ -122,11 +122,11 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         float4* dst = reinterpret_cast<float4*>(gen);
         for (uint32_t i = threadIdx.x; i < image_bytes / 16; i += kChainTcThreads) dst[i] = src[i];
         for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
-            sbzs[i] = a.bz[i] * 2.8853900817779268f;
+            sbzs[i] = a.bz[i];
             sb1[i] = a.b1[i];
             sb3[i] = a.b3[i];
         }
-        for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i] + 1.0f) * (1.0f / 3.0f);
+        for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i]) * (1.0f / 3.0f);
         for (int i = threadIdx.x; i < 256; i += kChainTcThreads) sWsig[i] = a.Wsig[i];
         if (threadIdx.x < 16) {
             sbmu[threadIdx.x] = a.bmu[threadIdx.x];
@@ -297,10 +297,9 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                                 const float lv[4] = {lq.x, lq.y, lq.z, lq.w};
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) {      // tanh, then (tanh + h_left + h_right) / 3
-                                    float e, r;
-                                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[4 * g + i]), 2.8853900817779268f, bv[i])));
-                                    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-                                    h[4 * g + i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                                    float t;
+                                    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(__uint_as_float(acc[4 * g + i]) + bv[i]));
+                                    h[4 * g + i] = fmaf(t, 1.0f / 3.0f, lv[i]);
                                 }
                             } else {
 #pragma unroll
