@@ -208,7 +208,7 @@ def run_evaluate(args, wl, weights, literal):
     from paper_1803_04209_b200 import binding, build, inputs
     build.build()
     torch.cuda.set_device(0)
-    n_hist = max(wl.window + 1, min(wl.history, 64))
+    n_hist = max(wl.window + 1, min(wl.history, 64), args.evaluate_offset)
     T = args.evaluate_steps
     trace = inputs.workload_trace(wl, n_hist + T)
     dev_all = torch.from_numpy(trace).cuda()
@@ -219,7 +219,7 @@ def run_evaluate(args, wl, weights, literal):
         ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, wl.S, precision=wl.precision, seed=2024,
                              flags=flags if not censor else flags & ~binding.FLAG_GRAPH)
         ctx.load_weights(weights)
-        for x in trace[:n_hist]:
+        for x in trace[max(0, n_hist - 64):n_hist]:
             ctx.push(x)
         cs = np.empty(T, dtype=np.int32)
         for t in range(T):
@@ -295,6 +295,8 @@ def main():
                     help="score the model's cutoff, a static cutoff, the Elfving 'order' cutoff and waiting for all "
                          "workers against the hindsight-best throughput on the workload's synthetic trace, then exit")
     ap.add_argument("--evaluate-steps", type=int, default=200)
+    ap.add_argument("--evaluate-offset", type=int, default=0,
+                    help="first step of the workload's trace that is scored (the steps a weight file was fitted on come before it)")
     ap.add_argument("--weights", default="", help="path of a weight file written by oracle/fit_elbo.py (npz); default: seeded random weights")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
