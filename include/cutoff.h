@@ -244,7 +244,10 @@ int64_t cutoff_launch_count(cutoff_ctx* ctx);
  * clipped to S and to the allocated pass buffers).  "order_stat_std": 1 = also compute the spread
  * of each order statistic (see cutoff_get_order_stat_std), 0 = do not (default); not available to a
  * context that holds only part of a decision's samples (UNSUPPORTED), nor once a graph has been
- * captured (STATE).  Errors: BAD_ARG, STATE, UNSUPPORTED. */
+ * captured (STATE).  "pair_emission": 1 = run the emission output layer (Section 3.1.3, x ~ N(I(z), J(z))) with
+ * tensor-core instructions that span two SMs, so that each SM loads only half of every weight tile (compact variant
+ * on a tensor-core precision only: UNSUPPORTED otherwise; same results as 0, the default, which is the faster one
+ * as measured); not once a graph has been captured (STATE).  Errors: BAD_ARG, STATE, UNSUPPORTED. */
 int cutoff_set_option(cutoff_ctx* ctx, const char* name, int64_t value);
 
 /* ---- test hooks ----------------------------------------------------------------------------

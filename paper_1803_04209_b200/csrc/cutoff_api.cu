@@ -12,6 +12,7 @@
 #include "kernels_model.cuh"
 #include "kernels_sort.cuh"
 #include "emit_tc.cuh"
+#include "emit_tc2.cuh"
 #include "chain_tc.cuh"
 #include "chain_tc32.cuh"
 #include "kernels_literal.cuh"
@@ -84,6 +85,8 @@ struct cutoff_ctx {
     CUtensorMap map_r{};            // TMA view of d_r [alloc_rows][H]
     CUtensorMap map_wi2{}, map_M{}, map_wj2{};
     bool use_tc = false;            // emission output layer on tensor cores
+    int pair_clusters = 0;          // clusters of two CTAs of the two-SM emission kernel that fit the GPU at once
+    bool pair_emission = false;     // option "pair_emission": run the output layer on pairs of SMs (slower as measured; off)
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
     bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
     bool chain_tcl = false;         // the literal variant's chain on tensor cores (D = 16, H in {64, 128, 192, 256})
@@ -380,6 +383,14 @@ void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
     a.b4 = c->m.b4; a.x = c->d_x; a.st = c->d_state;
     a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     a.sample_base = sample_base; a.count = count; a.N = c->N; a.H = c->H; a.ldx = c->ldx;
+    if (c->pair_emission && c->pair_clusters > 0 && count > tc::kBM) {
+        // pairs of SMs share a weight tile: 256 samples x 128 workers per cluster and tile
+        const int pair_tiles = ceil_div(c->N, tc::kBW) * ceil_div(count, 2 * tc::kBM);
+        const int clusters = pair_tiles < c->pair_clusters ? pair_tiles : c->pair_clusters;
+        tc::k_emit_tc2<<<2 * clusters, tc::kThreads, tc::kSmem2Bytes, c->stream>>>(c->map_v, c->map_w4, a);
+        c->launches += 1;
+        return;
+    }
     const int tiles = ceil_div(c->N, tc::kBW) * ceil_div(count, tc::kBM);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
     tc::k_emit_tc<<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(c->map_v, c->map_w4, a);
@@ -593,6 +604,7 @@ cudaError_t set_kernel_attributes(const cutoff_ctx* c) {
     if (e == cudaSuccess) e = allow_smem(k_enc_rnn_cluster, 200 * 1024);
     if (e != cudaSuccess || !c->use_tc) return e;
     e = allow_smem(tc::k_emit_tc, tc::kSmemBytes);
+    if (e == cudaSuccess) e = allow_smem(tc::k_emit_tc2, tc::kSmem2Bytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_gemm_relu_tc, tc::kSmemBytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_emit_dual_tc, tc::kDualSmemBytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc, 227 * 1024);
@@ -728,6 +740,21 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
         if (rc) return fail(rc);
     }
     CREATE_CHECK(set_kernel_attributes(c));
+    if (c->use_tc && !c->literal) {
+        // how many two-CTA clusters of the two-SM emission kernel the GPU can hold at once
+        cudaLaunchConfig_t lc{};
+        lc.gridDim = dim3(2 * c->sm_count);
+        lc.blockDim = dim3(tc::kThreads);
+        lc.dynamicSmemBytes = tc::kSmem2Bytes;
+        cudaLaunchAttribute at{};
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = 2; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+        lc.attrs = &at;
+        lc.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, tc::k_emit_tc2, &lc) == cudaSuccess && n > 0) c->pair_clusters = n;
+        else cudaGetLastError();
+    }
     CREATE_CHECK(cudaMallocHost(&c->h_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMallocHost(&c->h_state, sizeof(DevState)));
     CREATE_CHECK(cudaMemsetAsync(c->d_state, 0, sizeof(DevState), c->stream));
@@ -1476,6 +1503,13 @@ int cutoff_set_option(cutoff_ctx* c, const char* name, int64_t value) {
         if (value && c->cfg.total_samples > 0 && c->cfg.total_samples != c->S) return CUTOFF_ERR_UNSUPPORTED;
         if (c->graph_exec || c->graph_dev_exec) return CUTOFF_ERR_STATE;   // the captured graph has the other sort kernel in it
         c->want_std = value != 0;
+        return CUTOFF_OK;
+    }
+    if (std::strcmp(name, "pair_emission") == 0) {
+        if (value != 0 && value != 1) return CUTOFF_ERR_BAD_ARG;
+        if (value && (c->literal || !c->use_tc || c->pair_clusters == 0)) return CUTOFF_ERR_UNSUPPORTED;
+        if (c->graph_exec || c->graph_dev_exec) return CUTOFF_ERR_STATE;   // the captured graph has the other kernel in it
+        c->pair_emission = value != 0;
         return CUTOFF_OK;
     }
     if (std::strcmp(name, "pass_rows") == 0) {

@@ -731,3 +731,19 @@ def test_measured_pipe_rates_are_plausible():
     assert 1.0 <= r["minmax"] <= 2.1          # 64 lanes per SM per clock = 2 warp-instructions
     assert 0.5 <= r["shuffle"] <= 1.1         # 32 lanes per SM per clock
     assert 2.0 <= r["fma"] <= 4.1             # 128 lanes per SM per clock
+
+
+@pytest.mark.parametrize("name,S", [("n1024", 700), ("n2175", 300), ("n4096", 384)])
+def test_two_sm_emission_option_gives_the_same_draws(name, S):
+    # the output layer with tensor-core instructions that span two SMs (each SM loads half of every weight tile)
+    wl, gpu, orc, prec = make_pair(name, S=S, steps=inputs.WORKLOADS[name].window + 7)
+    ref = gpu.debug_samples(0, S)
+    gpu.set_option("pair_emission", 1)
+    got = gpu.debug_samples(0, S)
+    assert np.allclose(got, ref, rtol=1e-6, atol=1e-7)
+    assert_samples_close(got, orc.samples(np.arange(S)), TOL_X[prec])
+    assert_decision_close(gpu, orc.predict(), wl.N)
+    fp32 = binding.Cutoff(16, 4, 32, 1, 64)
+    with pytest.raises(binding.CutoffError) as e:
+        fp32.set_option("pair_emission", 1)
+    assert e.value.code == binding.ERR_UNSUPPORTED
