@@ -175,6 +175,21 @@ std::vector<TensorSpec> tensor_specs_literal(size_t N, size_t D, size_t H) {
     return v;
 }
 
+// Round to tf32 as the tensor cores will see the value (nearest, ties away from zero), kept as an fp32 bit pattern.
+float host_tf32(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    u = (u + 0x1000u) & 0xFFFFE000u;
+    std::memcpy(&f, &u, 4);
+    return f;
+}
+
+// Float index of element (row, col) inside one K-major operand slab of rows x 32 with 128-byte rows whose 16-byte
+// chunks are XOR-swizzled with the row index modulo 8 (the layout the tensor cores read from shared memory).
+size_t swz(size_t row, size_t col) {
+    return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
+}
+
 int next_pow2(int n) {
     int p = 1;
     while (p < n) p <<= 1;
@@ -853,16 +868,6 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     if (c->chain_tc) {
         // Operand tiles of the tensor-core chain as they will sit in shared memory: tf32 (nearest, ties
         // away), K-major rows of 32 values, 16-byte chunks XOR-swizzled with the row index modulo 8.
-        auto tf32 = [](float f) {
-            uint32_t u;
-            std::memcpy(&u, &f, 4);
-            u = (u + 0x1000u) & 0xFFFFE000u;
-            std::memcpy(&f, &u, 4);
-            return f;
-        };
-        auto at = [](size_t row, size_t col) {       // float index inside one slab of rows x 32
-            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
-        };
         std::vector<float> img(tc::chain_tc_image_floats(c->H), 0.0f);
         const float* wz = host.data() + off[8];      // [H][D]
         const float* w1 = host.data() + off[15];     // [H][D]
@@ -875,14 +880,14 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         float* t_w2 = t_wmu + H * 16;
         for (size_t n = 0; n < H; ++n)
             for (size_t k = 0; k < D; ++k) {
-                t_zw1[at(n, k)] = tf32(wz[n * D + k]);
-                t_zw1[at(n, 16 + k)] = tf32(w1[n * D + k]);
-                t_w3[at(n, k)] = tf32(w3[n * D + k]);
+                t_zw1[swz(n, k)] = host_tf32(wz[n * D + k]);
+                t_zw1[swz(n, 16 + k)] = host_tf32(w1[n * D + k]);
+                t_w3[swz(n, k)] = host_tf32(w3[n * D + k]);
             }
         for (size_t kb = 0; kb < H / 32; ++kb)
             for (size_t jj = 0; jj < 32; ++jj) {
-                for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
-                for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + at(o, jj)] = tf32(w2[o * H + kb * 32 + jj]);
+                for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + swz(d, jj)] = host_tf32(wmu[d * H + kb * 32 + jj]);
+                for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + swz(o, jj)] = host_tf32(w2[o * H + kb * 32 + jj]);
             }
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
@@ -890,16 +895,6 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     if (c->chain_tcl) {
         // Literal variant, D = 16: [Wz | Wg1] and [Wh1 | Wi1] as [H rows][32], Wmu, Wg2, Wh2 as H/32 K blocks of
         // [16 rows][32], Ws as [16 rows][32] (columns 16.. zero), all tf32 in the swizzled shared-memory layout.
-        auto tf32 = [](float f) {
-            uint32_t u;
-            std::memcpy(&u, &f, 4);
-            u = (u + 0x1000u) & 0xFFFFE000u;
-            std::memcpy(&f, &u, 4);
-            return f;
-        };
-        auto at = [](size_t row, size_t col) {
-            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
-        };
         std::vector<float> img(tc::chain_tcl_image_floats(c->H), 0.0f);
         const float* wz = host.data() + off[8];      // [H][D]
         const float* wg1 = host.data() + off[15];
@@ -913,34 +908,24 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         float* t_ws = t_second + 3 * H * 16;
         for (size_t n = 0; n < H; ++n)
             for (size_t k = 0; k < D; ++k) {
-                t_zg[at(n, k)] = tf32(wz[n * D + k]);
-                t_zg[at(n, 16 + k)] = tf32(wg1[n * D + k]);
-                t_hi[at(n, k)] = tf32(wh1[n * D + k]);
-                t_hi[at(n, 16 + k)] = tf32(wi1[n * D + k]);
+                t_zg[swz(n, k)] = host_tf32(wz[n * D + k]);
+                t_zg[swz(n, 16 + k)] = host_tf32(wg1[n * D + k]);
+                t_hi[swz(n, k)] = host_tf32(wh1[n * D + k]);
+                t_hi[swz(n, 16 + k)] = host_tf32(wi1[n * D + k]);
             }
         for (int t = 0; t < 3; ++t)
             for (size_t kb = 0; kb < H / 32; ++kb)
                 for (size_t jj = 0; jj < 32; ++jj)
                     for (size_t d = 0; d < D; ++d)
-                        t_second[t * H * 16 + kb * 16 * 32 + at(d, jj)] = tf32(second[t][d * H + kb * 32 + jj]);
+                        t_second[t * H * 16 + kb * 16 * 32 + swz(d, jj)] = host_tf32(second[t][d * H + kb * 32 + jj]);
         for (size_t o = 0; o < D; ++o)
-            for (size_t e = 0; e < D; ++e) t_ws[at(o, e)] = tf32(ws[o * D + e]);
+            for (size_t e = 0; e < D; ++e) t_ws[swz(o, e)] = host_tf32(ws[o * D + e]);
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
 
     if (c->chain_tc32) {
         // D = 32: six tiles of H x 32 tf32 values each -- Wz, W1, W3 as [H rows][32], Wmu and the two halves of W2 as
         // H/32 K blocks of [32 rows][32] -- in the swizzled shared-memory layout, staged by the kernel phase by phase
-        auto tf32 = [](float f) {
-            uint32_t u;
-            std::memcpy(&u, &f, 4);
-            u = (u + 0x1000u) & 0xFFFFE000u;
-            std::memcpy(&f, &u, 4);
-            return f;
-        };
-        auto at = [](size_t row, size_t col) {
-            return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
-        };
         const size_t tile = H * 32;
         std::vector<float> img(tc::chain_tc32_image_floats(c->H), 0.0f);
         const float* wz = host.data() + off[8];
@@ -950,16 +935,16 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         const float* w2 = host.data() + off[17];     // [64][H]: rows 0..31 mean, 32..63 log-variance
         for (size_t n = 0; n < H; ++n)
             for (size_t k = 0; k < 32; ++k) {
-                img[0 * tile + at(n, k)] = tf32(wz[n * 32 + k]);
-                img[1 * tile + at(n, k)] = tf32(w1[n * 32 + k]);
-                img[2 * tile + at(n, k)] = tf32(w3[n * 32 + k]);
+                img[0 * tile + swz(n, k)] = host_tf32(wz[n * 32 + k]);
+                img[1 * tile + swz(n, k)] = host_tf32(w1[n * 32 + k]);
+                img[2 * tile + swz(n, k)] = host_tf32(w3[n * 32 + k]);
             }
         for (size_t kb = 0; kb < H / 32; ++kb)
             for (size_t jj = 0; jj < 32; ++jj)
                 for (size_t d = 0; d < 32; ++d) {
-                    img[3 * tile + kb * 1024 + at(d, jj)] = tf32(wmu[d * H + kb * 32 + jj]);
-                    img[4 * tile + kb * 1024 + at(d, jj)] = tf32(w2[d * H + kb * 32 + jj]);
-                    img[5 * tile + kb * 1024 + at(d, jj)] = tf32(w2[(32 + d) * H + kb * 32 + jj]);
+                    img[3 * tile + kb * 1024 + swz(d, jj)] = host_tf32(wmu[d * H + kb * 32 + jj]);
+                    img[4 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[d * H + kb * 32 + jj]);
+                    img[5 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[(32 + d) * H + kb * 32 + jj]);
                 }
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }

@@ -6,7 +6,7 @@
 // H and J are standard deviations.  The guide is the one of kernels_model.cuh.
 //
 // The chain kernel ends with the first (affine) layer of I; the rest of the emission is three
-// matrix products over all samples (k_gemm_fma here, tc::k_gemm_tc on the tensor cores):
+// matrix products over all samples (k_gemm_fma here; tc::k_gemm_relu_tc and tc::k_emit_dual_tc on the tensor cores):
 //   I = u Wi2^T + bi2        r = relu(I Wj1^T + bj1)        x = I + softplus(r Wj2^T + bj2) * eps
 #pragma once
 #include "common.cuh"
