@@ -302,6 +302,42 @@ int cutoff_eval_trace(int device, const float* trace, int64_t n_steps, int32_t n
 int cutoff_order_baseline(int device, const float* trace, int64_t n_steps, int32_t n, int32_t ld, int32_t* cutoffs_out,
                           void* stream);
 
+/* ---- learning the model -----------------------------------------------------------------------------
+ * Section 3.1.3 fits the generative model p_theta and the guide q_phi together by stochastic gradient ascent on
+ *     ELBO = E_q [ log p_theta(x_{T-l:T}, z_{T-l:T}) - log q_phi(z_{T-l:T} | x_{T-l:T}) ],
+ * Section 4.1 names the optimiser: Adam with gradient clipping.  These calls are one training step's arithmetic for
+ * the compact networks, in fp32, on device buffers of the caller (the noise is an input: draw it as you like).
+ *
+ * The parameter vector is the tensors of the weight blob, in its order (Wxf Whf bf a0 Wxb Whb bb b0 Wz bz Wmu bmu
+ * Wsig bsig z0 W1 b1 W2 b2 W3 b3 W4 b4), back to back without the header: cutoff_fit_param_count floats.
+ *
+ * cutoff_elbo_grad: the one-sample reparameterised ELBO of each of `batch` windows -- z_t = mu_t + sigma_t eps_t,
+ * sum over the window's steps of log p(x_t | z_t) + log p(z_t | z_{t-1}) - log q(z_t | ...) with the densities of the
+ * mean / log-variance heads and the guide of Section 3.1.3; the latent before the window is z0, the RNNs start from
+ * a0 and b0 -- and the gradient of their SUM with respect to every parameter.
+ *   params  device, cutoff_fit_param_count floats
+ *   xhat    device, batch x (lag+1) x n_workers floats: normalised run-times (divided by twice the mean of the first
+ *           window, Section 3.1.3 last paragraph), oldest vector of a window first
+ *   eps     device, batch x (lag+1) x latent_dim floats: the standard-normal draws of the guide
+ *   elbo    device, batch floats, overwritten
+ *   grads   device, cutoff_fit_param_count floats, overwritten; NULL = forward pass only
+ *   workspace  device, at least cutoff_fit_workspace_bytes(...) bytes, contents undefined afterwards
+ * Only enqueues work on `stream`.  Every reduction runs in a fixed order: results are reproducible bit for bit.
+ *
+ * cutoff_adam_step: g = grad_scale * grads (e.g. -1/batch to minimise the negative mean ELBO); if ||g|| over all n
+ * entries exceeds clip_norm, g is scaled by clip_norm / ||g||; then Adam's step number t (1, 2, ...):
+ * m = beta1 m + (1-beta1) g, v = beta2 v + (1-beta2) g^2, params -= lr (m / (1-beta1^t)) / (sqrt(v / (1-beta2^t)) + eps).
+ * params, m, v: device, n floats, updated in place (m and v start at zero); norm_out: device, one float, receives ||g||
+ * before clipping; workspace: device, at least 2048 bytes.  Only enqueues.  Errors of both: BAD_ARG, CUDA. */
+int64_t cutoff_fit_param_count(int32_t n_workers, int32_t latent_dim, int32_t hidden);
+int64_t cutoff_fit_workspace_bytes(int32_t n_workers, int32_t latent_dim, int32_t hidden, int32_t lag, int32_t batch);
+int cutoff_elbo_grad(int device, int32_t n_workers, int32_t latent_dim, int32_t hidden, int32_t lag, int32_t batch,
+                     const float* params, const float* xhat, const float* eps, float* elbo, float* grads, void* workspace,
+                     size_t workspace_bytes, void* stream);
+int cutoff_adam_step(int device, int64_t n, float* params, const float* grads, float* m, float* v, int32_t t, float lr,
+                     float beta1, float beta2, float eps, float clip_norm, float grad_scale, float* norm_out, void* workspace,
+                     size_t workspace_bytes, void* stream);
+
 /* ---- allocation-free entry point ---------------------------------------------------------------
  * The paper has no counterpart for this call.  It serves programs that may not allocate device
  * memory at the time they need order statistics: a server that handed all of the GPU's memory to

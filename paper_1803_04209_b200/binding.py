@@ -34,6 +34,7 @@ EXPORTS = (
     "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
     "cutoff_debug_sort_values", "cutoff_predict_partial_async", "cutoff_partial_sums_device",
     "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates", "cutoff_eval_trace", "cutoff_order_baseline",
+    "cutoff_fit_param_count", "cutoff_fit_workspace_bytes", "cutoff_elbo_grad", "cutoff_adam_step",
     "cutoff_sorted_row_sums_static",
 )
 
@@ -104,6 +105,12 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_eval_trace": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, C.c_int32, vp, vp, vp, vp, vp,
                                         vp, vp]),
         "cutoff_order_baseline": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
+        "cutoff_fit_param_count": (C.c_int64, [C.c_int32, C.c_int32, C.c_int32]),
+        "cutoff_fit_workspace_bytes": (C.c_int64, [C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+        "cutoff_elbo_grad": (C.c_int, [C.c_int, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32, vp, vp, vp, vp, vp, vp,
+                                       C.c_size_t, vp]),
+        "cutoff_adam_step": (C.c_int, [C.c_int, C.c_int64, vp, vp, vp, vp, C.c_int32, C.c_float, C.c_float, C.c_float,
+                                       C.c_float, C.c_float, C.c_float, vp, vp, C.c_size_t, vp]),
         "cutoff_sorted_row_sums_static": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -409,6 +416,68 @@ def order_baseline(trace, stream: int | None = None):
     if rc < 0:
         raise CutoffError(rc, "cutoff_order_baseline")
     return out
+
+
+def flatten_weights(weights: dict) -> np.ndarray:
+    """The compact model's tensors in blob order as one fp32 vector (the parameter vector of the learning calls)."""
+    return np.concatenate([np.ascontiguousarray(weights[name], dtype=np.float32).reshape(-1) for name in TENSOR_ORDER])
+
+
+def unflatten_weights(flat: np.ndarray, N: int, D: int, H: int) -> dict:
+    out, o = {}, 0
+    for name in TENSOR_ORDER:
+        shape = tensor_shapes(N, D, H)[name]
+        n = int(np.prod(shape))
+        out[name] = np.asarray(flat[o:o + n], dtype=np.float32).reshape(shape).copy()
+        o += n
+    return out
+
+
+class Fitter:
+    """Training steps of the compact model on one GPU: device buffers owned here, arithmetic in the library."""
+
+    def __init__(self, N: int, D: int, H: int, lag: int, batch: int, weights: dict, device: int = 0):
+        import torch
+        self._lib = load_library()
+        self.N, self.D, self.H, self.lag, self.batch, self.device = N, D, H, lag, batch, device
+        dev = torch.device("cuda", device)
+        self.n = int(self._lib.cutoff_fit_param_count(N, D, H))
+        flat = flatten_weights(weights)
+        assert flat.size == self.n
+        self.params = torch.from_numpy(flat).to(dev)
+        self.grads = torch.zeros(self.n, dtype=torch.float32, device=dev)
+        self.m = torch.zeros_like(self.grads)
+        self.v = torch.zeros_like(self.grads)
+        self.elbo = torch.zeros(batch, dtype=torch.float32, device=dev)
+        self.norm = torch.zeros(1, dtype=torch.float32, device=dev)
+        ws = int(self._lib.cutoff_fit_workspace_bytes(N, D, H, lag, batch))
+        self.ws = torch.empty(max(ws, 4096), dtype=torch.uint8, device=dev)
+        self.t = 0
+
+    def elbo_grad(self, xhat, eps, want_grad: bool = True):
+        """xhat [batch, lag+1, N], eps [batch, lag+1, D]: contiguous fp32 CUDA tensors.  Returns (elbo, grads) tensors."""
+        import torch
+        rc = self._lib.cutoff_elbo_grad(self.device, self.N, self.D, self.H, self.lag, self.batch, self.params.data_ptr(),
+                                        xhat.data_ptr(), eps.data_ptr(), self.elbo.data_ptr(),
+                                        self.grads.data_ptr() if want_grad else None, self.ws.data_ptr(), self.ws.numel(),
+                                        torch.cuda.current_stream().cuda_stream)
+        if rc < 0:
+            raise CutoffError(rc, "cutoff_elbo_grad")
+        return self.elbo, self.grads
+
+    def adam_step(self, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, clip=10.0, grad_scale=None):
+        """One Adam step on the negative mean ELBO (grad_scale = -1/batch) with clipping by the global norm."""
+        import torch
+        self.t += 1
+        scale = -1.0 / self.batch if grad_scale is None else grad_scale
+        rc = self._lib.cutoff_adam_step(self.device, self.n, self.params.data_ptr(), self.grads.data_ptr(), self.m.data_ptr(),
+                                        self.v.data_ptr(), self.t, lr, beta1, beta2, eps, clip, scale, self.norm.data_ptr(),
+                                        self.ws.data_ptr(), self.ws.numel(), torch.cuda.current_stream().cuda_stream)
+        if rc < 0:
+            raise CutoffError(rc, "cutoff_adam_step")
+
+    def weights(self) -> dict:
+        return unflatten_weights(self.params.cpu().numpy(), self.N, self.D, self.H)
 
 
 def sorted_row_sums_static(x, sums, n: int | None = None, stream: int | None = None) -> int:

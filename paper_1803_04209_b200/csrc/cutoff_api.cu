@@ -20,6 +20,7 @@
 #include "chain_tc_literal.cuh"
 #include "pipe_rates.cuh"
 #include "kernels_eval.cuh"
+#include "fit_api.cuh"
 
 using namespace cutoff;
 
@@ -1737,6 +1738,57 @@ int cutoff_order_baseline(int device, const float* trace, int64_t n_steps, int32
     const cudaError_t err = cudaStreamSynchronize(s);
     cudaFree(d_work);
     return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
+}
+
+// ---- learning the model: ELBO, gradient, Adam -------------------------------------------------------------------
+
+int64_t cutoff_fit_param_count(int32_t n_workers, int32_t latent_dim, int32_t hidden) {
+    if (n_workers < 1 || latent_dim < 1 || hidden < 1) return 0;
+    return fit::layout(n_workers, latent_dim, hidden).off[fit::kTensors];
+}
+
+int64_t cutoff_fit_workspace_bytes(int32_t n_workers, int32_t latent_dim, int32_t hidden, int32_t lag, int32_t batch) {
+    if (n_workers < 1 || latent_dim < 1 || hidden < 1 || lag < 0 || batch < 1) return 0;
+    return static_cast<int64_t>(sizeof(float)) * fit::workspace_floats(n_workers, latent_dim, hidden, lag + 1, batch);
+}
+
+int cutoff_elbo_grad(int device, int32_t n_workers, int32_t latent_dim, int32_t hidden, int32_t lag, int32_t batch,
+                     const float* params, const float* xhat, const float* eps, float* elbo, float* grads, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    if (device < 0 || n_workers < 1 || n_workers > 4096 || latent_dim < 1 || latent_dim > 64 || hidden < 1 || hidden > 1024 ||
+        lag < 0 || lag > 255 || batch < 1 || batch > 65535 || !params || !xhat || !eps || !elbo || !workspace)
+        return CUTOFF_ERR_BAD_ARG;
+    if (workspace_bytes < static_cast<size_t>(cutoff_fit_workspace_bytes(n_workers, latent_dim, hidden, lag, batch)))
+        return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    fit::elbo_grad(n_workers, latent_dim, hidden, lag + 1, batch, params, xhat, eps, elbo, grads,
+                   static_cast<float*>(workspace), static_cast<cudaStream_t>(stream));
+    return cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
+}
+
+int cutoff_adam_step(int device, int64_t n, float* params, const float* grads, float* m, float* v, int32_t t, float lr,
+                     float beta1, float beta2, float eps, float clip_norm, float grad_scale, float* norm_out, void* workspace,
+                     size_t workspace_bytes, void* stream) {
+    constexpr int kParts = 256;
+    if (device < 0 || n < 1 || !params || !grads || !m || !v || t < 1 || !(lr > 0.f) || !(beta1 >= 0.f && beta1 < 1.f) ||
+        !(beta2 >= 0.f && beta2 < 1.f) || !(eps > 0.f) || !(clip_norm > 0.f) || !norm_out || !workspace ||
+        workspace_bytes < kParts * sizeof(double))
+        return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    double* partial = static_cast<double*>(workspace);
+    const int64_t want = (n + fit::kNormThreads - 1) / fit::kNormThreads;
+    const int parts = static_cast<int>(want < kParts ? want : kParts);
+    fit::k_sumsq_partial<<<parts, fit::kNormThreads, 0, s>>>(grads, n, grad_scale, partial);
+    fit::k_norm_finish<<<1, 32, 0, s>>>(partial, parts, norm_out);
+    const float corr1 = 1.f - std::pow(beta1, static_cast<float>(t)), corr2 = 1.f - std::pow(beta2, static_cast<float>(t));
+    fit::k_adam<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(params, grads, m, v, n, grad_scale, norm_out, clip_norm, lr,
+                                                                      beta1, beta2, eps, corr1, corr2);
+    return cudaGetLastError() == cudaSuccess ? CUTOFF_OK : CUTOFF_ERR_CUDA;
 }
 
 }  // extern "C"
