@@ -201,6 +201,41 @@ def load_weight_file(path: str) -> dict:
         return {k: np.ascontiguousarray(z[k], dtype=np.float32) for k in z.files if not k.startswith("_")}
 
 
+def fit_on_gpu(args, wl, weights):
+    """Section 4.1: Adam with gradient clipping on the ELBO of Section 3.1.3, every step's arithmetic in the library.
+    Trains on the windows of the trace's first --evaluate-offset steps; returns (weights, report)."""
+    import torch
+    from paper_1803_04209_b200 import binding, inputs
+    n_train = max(args.evaluate_offset, 4 * wl.window + 64)
+    trace = inputs.workload_trace(wl, n_train).astype(np.float64)
+    scale = 2.0 * float(trace[: wl.window].mean())                  # the run-time normaliser: twice the first window's mean
+    norm = torch.from_numpy((trace / scale).astype(np.float32)).cuda()
+    n_win = n_train - wl.window + 1
+    batch = 64
+    fitter = binding.Fitter(wl.N, wl.D, wl.H, wl.lag, batch, weights)
+    gen = torch.Generator(device="cuda").manual_seed(0)
+    offs = torch.arange(wl.window, device="cuda")
+    first = last = None
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for it in range(args.fit_steps):
+        idx = torch.randint(0, n_win, (batch,), device="cuda", generator=gen)
+        xhat = norm[idx[:, None] + offs[None, :]].contiguous()       # [batch, window, N]
+        eps = torch.randn((batch, wl.window, wl.D), device="cuda", generator=gen)
+        elbo, _ = fitter.elbo_grad(xhat, eps)
+        fitter.adam_step(lr=2e-3, clip=10.0)
+        if it == 0 or it == args.fit_steps - 1:
+            val = float(elbo.mean().item())
+            first = val if it == 0 else first
+            last = val
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    report = {"steps": args.fit_steps, "batch_windows": batch, "train_trace_steps": n_train, "seconds": round(sec, 2),
+              "steps_per_second": round(args.fit_steps / sec, 1), "elbo_per_window_first": first, "elbo_per_window_last": last,
+              "how": "cutoff_elbo_grad + cutoff_adam_step per step (fp32, lr 2e-3, clip 10), windows and noise drawn with torch on the GPU"}
+    return fitter.weights(), report
+
+
 def run_evaluate(args, wl, weights, literal):
     """Fig. 2's comparison on the workload's synthetic trace: throughput achieved by each cutoff rule relative to
     the hindsight-best throughput of every step.  All scoring runs in the library's kernels."""
@@ -208,6 +243,11 @@ def run_evaluate(args, wl, weights, literal):
     from paper_1803_04209_b200 import binding, build, inputs
     build.build()
     torch.cuda.set_device(0)
+    fit_report = None
+    if args.fit_steps > 0:
+        if literal:
+            raise SystemExit("--fit-steps fits the compact networks only")
+        weights, fit_report = fit_on_gpu(args, wl, weights)
     n_hist = max(wl.window + 1, min(wl.history, 64), args.evaluate_offset)
     T = args.evaluate_steps
     trace = inputs.workload_trace(wl, n_hist + T)
@@ -254,10 +294,10 @@ def run_evaluate(args, wl, weights, literal):
                         "total_fraction_of_best": float(ach.sum() / best.sum()),
                         "mean_step_seconds": float(res["step_time"][m].double().mean()),
                         "mean_cutoff": float(np.mean(rules[name]))}
-    fitted = bool(args.weights)
+    fitted = bool(args.weights) or fit_report is not None
     line = {"evaluate": {"workload": wl.name, "variant": args.variant, "N": wl.N, "S": wl.S, "steps": T,
-                         "history_steps": n_hist,
-                         "weights": args.weights if fitted else "seeded random initialisation with hand-set bias offsets",
+                         "history_steps": n_hist, "fit": fit_report,
+                         "weights": (args.weights or "fitted on the GPU in this run") if fitted else "seeded random initialisation with hand-set bias offsets",
                          "note": ("model rows use fitted weights" if fitted else
                                   "the model rows are a plumbing check only: the weights are not fitted to this trace"),
                          "hindsight_mean_cutoff": float(res["best_c"].double().mean()),
@@ -297,6 +337,9 @@ def main():
     ap.add_argument("--evaluate-steps", type=int, default=200)
     ap.add_argument("--evaluate-offset", type=int, default=0,
                     help="first step of the workload's trace that is scored (the steps a weight file was fitted on come before it)")
+    ap.add_argument("--fit-steps", type=int, default=0,
+                    help="with --evaluate: first fit the weights on the GPU (the library's ELBO gradient and Adam calls) for "
+                         "this many steps of 64 windows on the trace before --evaluate-offset")
     ap.add_argument("--weights", default="", help="path of a weight file written by oracle/fit_elbo.py (npz); default: seeded random weights")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "cuda":
