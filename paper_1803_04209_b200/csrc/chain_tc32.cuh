@@ -88,11 +88,11 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc32(ChainTc32Args
     const int epi_thread = threadIdx.x - 32;               // 0..511 for the epilogue warps
 
     for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
-        sbzs[i] = a.bz[i] * 2.8853900817779268f;
+        sbzs[i] = a.bz[i];
         sb1[i] = a.b1[i];
         sb3[i] = a.b3[i];
     }
-    for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i] + 1.0f) * (1.0f / 3.0f);
+    for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i]) * (1.0f / 3.0f);
     for (int i = threadIdx.x; i < 1024; i += kChainTcThreads) sWsig[i] = a.Wsig[i];
     if (threadIdx.x < 32) {
         sbmu[threadIdx.x] = a.bmu[threadIdx.x];
@@ -238,10 +238,9 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc32(ChainTc32Args
                         const float lv[8] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
-                            float e, r;
-                            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
-                            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-                            h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                            float t;                                   // tanh by the hardware instruction (chain_tc.cuh)
+                            asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(__uint_as_float(acc[i]) + bv[i]));
+                            h[i] = fmaf(t, 1.0f / 3.0f, lv[i]);
                         }
                     } else {
 #pragma unroll

@@ -67,11 +67,11 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc_literal(ChainTc
     const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u + 2048u;
     const uint32_t t_act = base + image_bytes;                    // Z0, Z1, then 4 hidden-chunk buffers: 6 x 16 KB
     // fp32 side tables
-    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz * 2 log2(e)
+    float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz
     float* sbg1 = sbzs + H;
     float* sbh1 = sbg1 + H;
     float* sbi1 = sbh1 + H;
-    float* slr = sbi1 + H;                   // [W][H]  (h_left + h_right + 1) / 3
+    float* slr = sbi1 + H;                   // [W][H]  (h_left + h_right) / 3
     float* sWsig = slr + W * H;              // [16][16]
     float* sWl = sWsig + 256;                // [16][16]
     float* sbmu = sWl + 256;
@@ -94,12 +94,12 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc_literal(ChainTc
         float4* dst = reinterpret_cast<float4*>(gen);
         for (uint32_t i = threadIdx.x; i < image_bytes / 16; i += kChainTcThreads) dst[i] = src[i];
         for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
-            sbzs[i] = a.bz[i] * 2.8853900817779268f;
+            sbzs[i] = a.bz[i];
             sbg1[i] = a.bg1[i];
             sbh1[i] = a.bh1[i];
             sbi1[i] = a.bi1[i];
         }
-        for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i] + 1.0f) * (1.0f / 3.0f);
+        for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i]) * (1.0f / 3.0f);
         for (int i = threadIdx.x; i < 256; i += kChainTcThreads) {
             sWsig[i] = a.Wsig[i];
             sWl[i] = a.Wl[i];
@@ -279,10 +279,9 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc_literal(ChainTc
                             const float lv[8] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
 #pragma unroll
                             for (int i = 0; i < 8; ++i) {          // tanh, then (tanh + h_left + h_right) / 3
-                                float e, r;
-                                asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(acc[i]), 2.8853900817779268f, bv[i])));
-                                asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
-                                h[i] = fmaf(r, -2.0f / 3.0f, lv[i]);
+                                float t;                                   // tanh by the hardware instruction (chain_tc.cuh)
+                                asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(__uint_as_float(acc[i]) + bv[i]));
+                                h[i] = fmaf(t, 1.0f / 3.0f, lv[i]);
                             }
                         } else if (ph < ph_emit) {
 #pragma unroll
