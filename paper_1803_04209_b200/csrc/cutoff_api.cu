@@ -91,6 +91,7 @@ struct cutoff_ctx {
     bool chain_tc = false;          // per-sample chain on tensor cores as well (D = 16, H in {64, 128, 192, 256})
     bool chain_tc32 = false;        // the same for D = 32, H <= 512 (weights staged phase by phase)
     bool chain_tcl = false;         // the literal variant's chain on tensor cores (D = 16, H in {64, 128, 192, 256})
+    bool chain_tcl32 = false;       // the same for D = 32, H <= 512 (weights staged phase by phase)
     float* d_chain_image = nullptr; // swizzled tf32 operand tiles of the chain
 
     float* h_stage = nullptr;       // pinned [N]
@@ -306,12 +307,18 @@ void launch_chain_tc32(cutoff_ctx* c, uint32_t sample_base, int count) {
     const ModelDev& m = c->m;
     a.image = c->d_chain_image;
     a.bz = m.bz; a.b1 = m.b1; a.b3 = m.b3; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig; a.b2 = m.b2; a.z0 = m.z0;
+    if (c->chain_tcl32) {
+        const LiteralDev& l = c->lit;
+        a.b1 = l.bg1; a.b3 = l.bh1; a.b2 = nullptr;
+        a.bi1 = l.bi1; a.bg2 = l.bg2; a.bh2 = l.bh2; a.Wl = l.Wl; a.bl = l.bl; a.bs = l.bs;
+    }
     a.hlr = c->d_hlr; a.st = c->d_state;
     a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.round_v = 1; a.v_out = c->d_v;
     const int tiles = ceil_div(count, 128);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    tc::k_chain_tc32<<<grid, tc::kChainTcThreads, tc::chain_tc32_smem_bytes(c->H, c->W), c->stream>>>(a);
+    if (c->chain_tcl32) tc::k_chain_tc32<true><<<grid, tc::kChainTcThreads, tc::chain_tc32_smem_bytes(c->H, c->W, true), c->stream>>>(a);
+    else tc::k_chain_tc32<false><<<grid, tc::kChainTcThreads, tc::chain_tc32_smem_bytes(c->H, c->W), c->stream>>>(a);
     c->launches += 1;
 }
 
@@ -341,6 +348,7 @@ void launch_chain_tc_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
 
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
     if (c->chain_tcl) { launch_chain_tc_literal(c, sample_base, count); return; }
+    if (c->chain_tcl32) { launch_chain_tc32(c, sample_base, count); return; }
     if (c->literal) {
         switch (c->D) {
             case 4: launch_chain_literal_t<4>(c, sample_base, count); break;
@@ -624,7 +632,8 @@ cudaError_t set_kernel_attributes(const cutoff_ctx* c) {
     if (e == cudaSuccess) e = allow_smem(tc::k_gemm_relu_tc, tc::kSmemBytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_emit_dual_tc, tc::kDualSmemBytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc, 227 * 1024);
-    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32<false>, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32<true>, 227 * 1024);
     if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc_literal, 227 * 1024);
     return e;
 }
@@ -712,6 +721,8 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
                    tc::chain_tcl_smem_bytes(c->H, c->W) <= 227 * 1024;
     c->chain_tc32 = !c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
                     (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W) <= 227 * 1024;
+    c->chain_tcl32 = c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
+                     (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W, true) <= 227 * 1024;
 
     size_t blob_floats = 0;
     for (const auto& t : c->literal ? tensor_specs_literal(c->N, c->D, c->H) : tensor_specs(c->N, c->D, c->H))
@@ -733,6 +744,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     if (c->chain_tc32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H)));
     if (c->chain_tcl) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tcl_image_floats(c->H)));
+    if (c->chain_tcl32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H, true)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_mask, c->N));
@@ -947,6 +959,27 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
                     img[4 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[d * H + kb * 32 + jj]);
                     img[5 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[(32 + d) * H + kb * 32 + jj]);
                 }
+        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
+    }
+
+    if (c->chain_tcl32) {
+        // Literal variant, D = 32: Wz, Wg1, Wh1, Wi1 as [H rows][32]; Wmu, Wg2, Wh2 as H/32 K blocks of [32 rows][32];
+        // Ws as [32 rows][32]; all tf32 in the swizzled shared-memory layout, staged by the kernel phase by phase.
+        const size_t tile = H * 32;
+        std::vector<float> img(tc::chain_tc32_image_floats(c->H, true), 0.0f);
+        const float* first[4] = {host.data() + off[8], host.data() + off[15], host.data() + off[19], host.data() + off[27]};   // Wz Wg1 Wh1 Wi1: [H][32]
+        const float* second[3] = {host.data() + off[10], host.data() + off[17], host.data() + off[21]};                       // Wmu Wg2 Wh2: [32][H]
+        const float* ws = host.data() + off[25];                                                                              // [32][32]
+        for (int t = 0; t < 4; ++t)
+            for (size_t n = 0; n < H; ++n)
+                for (size_t k = 0; k < 32; ++k) img[t * tile + swz(n, k)] = host_tf32(first[t][n * 32 + k]);
+        for (int t = 0; t < 3; ++t)
+            for (size_t kb = 0; kb < H / 32; ++kb)
+                for (size_t jj = 0; jj < 32; ++jj)
+                    for (size_t d = 0; d < 32; ++d)
+                        img[(4 + t) * tile + kb * 1024 + swz(d, jj)] = host_tf32(second[t][d * H + kb * 32 + jj]);
+        for (size_t o = 0; o < 32; ++o)
+            for (size_t e = 0; e < 32; ++e) img[7 * tile + swz(o, e)] = host_tf32(ws[o * 32 + e]);
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
 
