@@ -3,5 +3,5 @@
 `binding` wraps libcutoff.so (hand-written sm_100a CUDA kernels), `build` compiles it in-tree,
 `inputs` draws the seeded synthetic weights and run-time traces.
 """
-from . import inputs  # noqa: F401
+from . import binding, inputs  # noqa: F401
 from .binding import Cutoff, CutoffError, debug_normals, load_library, pack_weights  # noqa: F401

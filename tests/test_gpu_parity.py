@@ -747,3 +747,39 @@ def test_two_sm_emission_option_gives_the_same_draws(name, S):
     with pytest.raises(binding.CutoffError) as e:
         fp32.set_option("pair_emission", 1)
     assert e.value.code == binding.ERR_UNSUPPORTED
+
+
+def test_sharded_decision_all_reduces_the_librarys_own_array_under_nccl():
+    # one rank, NCCL: the path bench.py takes with several GPUs -- the partial sums stay in the library's device
+    # array, NCCL reduces them in place on the context's stream, the decision is finished from there
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_1803_04209_b200 import sharding
+    wl = inputs.WORKLOADS["n128"]
+    S = 1024
+    stream = torch.cuda.current_stream()
+    w = inputs.workload_weights(wl)
+    trace = inputs.workload_trace(wl, 8)
+    cfg = sharding.shard_config(0, 1, S)
+    ctx = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, cfg["n_samples"], precision=wl.precision, seed=SEED,
+                         stream=stream.cuda_stream, sample_offset=cfg["sample_offset"], total_samples=cfg["total_samples"])
+    ref = binding.Cutoff(wl.N, wl.D, wl.H, wl.lag, S, precision=wl.precision, seed=SEED)
+    for c in (ctx, ref):
+        c.load_weights(w)
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                            device_id=torch.device("cuda", 0))
+    try:
+        shared = sharding.ShardedDecision(ctx, device="cuda")
+        assert shared.predict() == (binding.WARMUP, wl.N)
+        for x in trace:
+            ctx.push(x)
+            ref.push(x)
+        for _ in range(3):
+            assert shared.predict() == ref.predict()
+            assert np.array_equal(ctx.get_stats()[0], ref.get_stats()[0])
+    finally:
+        dist.destroy_process_group()
