@@ -236,6 +236,15 @@ int cutoff_set_timing(cutoff_ctx* ctx, int on);
  * multiply-adds, each from 32 warps per SM running independent chains.  Allocates and frees a few KB of
  * device memory, synchronises the device.  Errors: BAD_ARG, NOMEM, CUDA. */
 int cutoff_measure_pipe_rates(int device, float* rates_out);
+
+/* cutoff_measure_operand_stream: the rate, in GB/s over the whole device, at which all SMs together can bring
+ * operand tiles from L2 into shared memory with the copies the emission output layer (Section 3.1.3,
+ * x ~ N(I(z), J(z))) issues: per K block three tensor-map boxes of 128 rows x 128 bytes into a ring of four
+ * stages, one CTA per SM, nothing consuming the data.  gbs_out (host, 2 floats): [0] from a 2 MB matrix that
+ * every SM re-reads (the weights' case), [1] from a 64 MB matrix (the hidden vectors' case).  A micro-benchmark
+ * of about 1 ms per case; the paper has no counterpart.  Allocates and frees 64 MB of device memory,
+ * synchronises the device.  Errors: BAD_ARG, NOMEM, CUDA, TIMEOUT (a copy did not land within its bounded wait). */
+int cutoff_measure_operand_stream(int device, float* gbs_out);
 int cutoff_get_timing(cutoff_ctx* ctx, float* ms, int cap);
 const char* cutoff_stage_name(int i);
 int64_t cutoff_launch_count(cutoff_ctx* ctx);

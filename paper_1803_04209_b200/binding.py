@@ -33,7 +33,7 @@ EXPORTS = (
     "cutoff_get_timing", "cutoff_stage_name", "cutoff_launch_count", "cutoff_set_option",
     "cutoff_debug_normals", "cutoff_debug_samples", "cutoff_debug_window", "cutoff_debug_sort",
     "cutoff_debug_sort_values", "cutoff_predict_partial_async", "cutoff_partial_sums_device",
-    "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates", "cutoff_eval_trace", "cutoff_order_baseline",
+    "cutoff_decide_from_device_sums", "cutoff_measure_pipe_rates", "cutoff_measure_operand_stream", "cutoff_eval_trace", "cutoff_order_baseline",
     "cutoff_fit_param_count", "cutoff_fit_workspace_bytes", "cutoff_elbo_grad", "cutoff_adam_step",
     "cutoff_sorted_row_sums_static",
 )
@@ -102,6 +102,7 @@ def load_library(path: str | None = None) -> C.CDLL:
         "cutoff_partial_sums_device": (C.c_int, [vp, C.POINTER(vp)]),
         "cutoff_decide_from_device_sums": (C.c_int, [vp, vp, i32p]),
         "cutoff_measure_pipe_rates": (C.c_int, [C.c_int, f32p]),
+        "cutoff_measure_operand_stream": (C.c_int, [C.c_int, f32p]),
         "cutoff_eval_trace": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, C.c_int32, vp, vp, vp, vp, vp,
                                         vp, vp]),
         "cutoff_order_baseline": (C.c_int, [C.c_int, vp, C.c_int64, C.c_int32, C.c_int32, vp, vp]),
@@ -376,6 +377,16 @@ def measure_pipe_rates(device: int = 0) -> dict:
     if rc < 0:
         raise CutoffError(rc, "cutoff_measure_pipe_rates")
     return {"minmax": float(out[0]), "shuffle": float(out[1]), "fma": float(out[2])}
+
+
+def measure_operand_stream(device: int = 0) -> dict:
+    """Measured rate (GB/s, whole device) of the emission kernel's operand copies L2 -> shared memory."""
+    lib = load_library()
+    out = (C.c_float * 2)()
+    rc = lib.cutoff_measure_operand_stream(device, out)
+    if rc < 0:
+        raise CutoffError(rc, "cutoff_measure_operand_stream")
+    return {"weights_2mb": float(out[0]), "hidden_64mb": float(out[1])}
 
 
 def eval_trace(trace, cutoffs=None, want_static: bool = True, stream: int | None = None) -> dict:

@@ -383,7 +383,7 @@ int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t r
         cudaDriverEntryPointQueryResult q;
         CU_CHECK(c, cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
         if (!fn || q != cudaDriverEntryPointSuccess) {
-            c->last_error = "cuTensorMapEncodeTiled is not available from this driver";
+            if (c) c->last_error = "cuTensorMapEncodeTiled is not available from this driver";
             return CUTOFF_ERR_CUDA;
         }
         encode = reinterpret_cast<EncodeFn>(fn);
@@ -396,7 +396,7 @@ int make_tile_map(cutoff_ctx* c, CUtensorMap* map, const float* base, uint64_t r
                               elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
-        c->last_error = "cuTensorMapEncodeTiled failed with code " + std::to_string(static_cast<int>(r));
+        if (c) c->last_error = "cuTensorMapEncodeTiled failed with code " + std::to_string(static_cast<int>(r));
         return CUTOFF_ERR_CUDA;
     }
     return CUTOFF_OK;
@@ -1435,6 +1435,58 @@ int cutoff_measure_pipe_rates(int device, float* rates_out) {
     }
     cudaFree(d_cycles);
     cudaFree(d_sink);
+    return rc;
+}
+
+int cutoff_measure_operand_stream(int device, float* gbs_out) {
+    if (device < 0 || !gbs_out) return CUTOFF_ERR_BAD_ARG;
+    cutoff_ctx* none = nullptr;
+    DeviceGuard guard(device);
+    CU_CHECK(none, guard.err);
+    cudaDeviceProp prop;
+    CU_CHECK(none, cudaGetDeviceProperties(&prop, device));
+    const int sms = prop.multiProcessorCount;
+    CU_CHECK(none, cudaFuncSetAttribute(k_operand_stream, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        static_cast<int>(kStreamSmemBytes)));
+    constexpr int kCols = 256;
+    const int rows_of[2] = {2048, 65536};                // 2 MB that every SM re-reads; 64 MB
+    float* d_src = nullptr;
+    int* d_err = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaMalloc(&d_src, sizeof(float) * rows_of[1] * kCols) != cudaSuccess) return CUTOFF_ERR_NOMEM;
+    int rc = CUTOFF_OK;
+    if (cudaMalloc(&d_err, sizeof(int)) != cudaSuccess) rc = CUTOFF_ERR_NOMEM;
+    if (rc == CUTOFF_OK && (cudaMemset(d_src, 0, sizeof(float) * rows_of[1] * kCols) != cudaSuccess ||
+                            cudaMemset(d_err, 0, sizeof(int)) != cudaSuccess || cudaEventCreate(&e0) != cudaSuccess ||
+                            cudaEventCreate(&e1) != cudaSuccess))
+        rc = CUTOFF_ERR_CUDA;
+    for (int which = 0; which < 2 && rc == CUTOFF_OK; ++which) {
+        CUtensorMap map;
+        rc = make_tile_map(nullptr, &map, d_src, rows_of[which], kCols);
+        if (rc != CUTOFF_OK) break;
+        const int iters = static_cast<int>((4096ll << 20) / sms / kStreamStageBytes);    // 4 GB per launch in all
+        float best = 0.0f;
+        for (int rep = 0; rep < 3; ++rep) {              // the first repetition fills the L2 and warms the clocks up
+            cudaEventRecord(e0);
+            k_operand_stream<<<sms, 32, kStreamSmemBytes>>>(map, rows_of[which], kCols / 32, iters, d_err);
+            cudaEventRecord(e1);
+            float ms = 0.0f;
+            if (cudaEventSynchronize(e1) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.0f) {
+                rc = CUTOFF_ERR_CUDA;
+                break;
+            }
+            const float gbs = static_cast<float>(static_cast<double>(iters) * kStreamStageBytes * sms / (ms * 1e6));
+            if (rep > 0 && gbs > best) best = gbs;
+        }
+        gbs_out[which] = best;
+    }
+    int h_err = 0;
+    if (rc == CUTOFF_OK && cudaMemcpy(&h_err, d_err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) rc = CUTOFF_ERR_CUDA;
+    if (rc == CUTOFF_OK && h_err) rc = CUTOFF_ERR_TIMEOUT;
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(d_src);
+    cudaFree(d_err);
     return rc;
 }
 

@@ -733,6 +733,17 @@ def test_measured_pipe_rates_are_plausible():
     assert 2.0 <= r["fma"] <= 4.1             # 128 lanes per SM per clock
 
 
+def test_measured_operand_stream_is_plausible():
+    # all SMs together, L2 -> shared memory: above what HBM alone could feed, below 64 bytes per clock per SM x 2
+    r = binding.measure_operand_stream(0)
+    assert 4000.0 <= r["hidden_64mb"] <= 40000.0
+    assert 4000.0 <= r["weights_2mb"] <= 40000.0
+    assert r["weights_2mb"] >= 0.8 * r["hidden_64mb"]
+    # a second call gives about the same figures (the first repetition of each is a warm-up)
+    r2 = binding.measure_operand_stream(0)
+    assert abs(r2["hidden_64mb"] - r["hidden_64mb"]) <= 0.2 * r["hidden_64mb"]
+
+
 @pytest.mark.parametrize("name,S", [("n1024", 700), ("n2175", 300), ("n4096", 384)])
 def test_two_sm_emission_option_gives_the_same_draws(name, S):
     # the output layer with tensor-core instructions that span two SMs (each SM loads half of every weight tile)
