@@ -1,5 +1,10 @@
-// Per-sample chain (guide steps, transition, emission hidden layer) on the tcgen05 tensor cores,
-// for latent size 16 and hidden width 64..256, operands in tf32.
+// Per-sample chain (guide steps, transition, first emission layer) on the tcgen05 tensor cores,
+// for latent size 16 and hidden width 64..256, operands in tf32.  One kernel template serves both model
+// variants: the compact one (transition = one hidden layer with a [mean | logvar] head, then the emission's
+// hidden layer v) and the networks as Section 3.1.3 prints them (LITERAL: gated transition
+//      g = sigmoid(Wg2 relu(Wg1 z + bg1) + bg2)        h = Wh2 relu(Wh1 z + bh1) + bh2
+//      G = (1 - g) * (Wl z + bl) + g * h               H = softplus(Ws relu(G) + bs)        z' = G + H * eps
+// then the affine first layer of the emission mean, u = Wi1 z' + bi1).
 //
 // A CTA walks over tiles of 128 samples; sample r of the tile is TMEM lane r.  Every layer pair
 //      hidden = act(A z + a)          (M=128, N=H, K=16)
@@ -8,14 +13,17 @@
 // epilogue warps read them 64 hidden units ("chunk") at a time, apply bias and activation, round
 // to tf32 and store the chunk as two K-major, 128-byte-swizzled A operand tiles in the buffer of
 // the tile's slot; the MMA warp multiplies that chunk with the matching K blocks of B while the
-// epilogue produces the same chunk of the other tile in flight.  The second result (mu, or mean | logvar) is read back by all
-// epilogue warps, which draw the noise, form the next latent and store it as the next A operand.
-// The last layer's hidden vector v goes to global memory for the emission output GEMM.
+// epilogue produces the same chunk of the other tile in flight.  The second result (mu; mean | logvar; gate;
+// proposal) is read back by all epilogue warps, which draw the noise, form the next latent and store it as the
+// next A operand.  In the literal variant the proposal's result is combined with the gate and the linear map
+// (computed by the epilogue threads from the latent tile) into G, relu(G) then takes the place of the latent
+// tile and one more small product with Ws gives the scale.
+// The last layer's hidden vector (v, or u) goes to global memory for the emission output GEMMs.
 //
 // All weight operands live in shared memory for the whole kernel: the host prepares their
 // swizzled image once, the CTA copies it in at start.  Latent rows are 128 bytes wide (32 tf32)
-// although K = 16: Wz and W1 share one tile (columns 0..15 and 16..31), so the MMA for the
-// transition simply starts 64 bytes into the rows.
+// although K = 16: two first-layer matrices share one tile (columns 0..15 and 16..31: [Wz | W1], or
+// [Wz | Wg1] and [Wh1 | Wi1]), so the MMA for the second of them simply starts 64 bytes into the rows.
 //
 // Warp 0 issues the MMAs and owns TMEM; warps 1..16 are the epilogue: warp w serves TMEM lanes
 // 32*(w%4).. and column group cg = (w-1)/4: 16 of each chunk's 64 columns and the latent
@@ -32,21 +40,29 @@ constexpr int kChainTcThreads = (1 + kChainEpiWarps) * 32;
 constexpr int kChainD = 16;
 
 struct ChainTcArgs {
-    const float* image;         // swizzled operand tiles: [Wz|W1] (H x 32), W3 (H x 32), Wmu (H/32 x 16 x 32), W2 (H/32 x 32 x 32)
+    // swizzled operand tiles.  compact: [Wz|W1] (H x 32), W3 (H x 32), Wmu (H/32 x 16 x 32), W2 (H/32 x 32 x 32);
+    // literal: [Wz|Wg1] (H x 32), [Wh1|Wi1] (H x 32), Wmu, Wg2, Wh2 (H/32 x 16 x 32 each), Ws (16 x 32)
+    const float* image;
+    // compact: b1, b3 = biases of the transition's and the emission's hidden layer, b2 = [mean | logvar] bias (32);
+    // literal: b1 = bg1, b3 = bh1, b2 unused
     const float *bz, *b1, *b3, *bmu, *bsig, *Wsig, *b2, *z0;
+    const float *bi1, *bg2, *bh2, *Wl, *bl, *bs;       // literal variant only
     const float* hlr;           // [2][W][H] h_left, h_right
     DevState* st;
     NoiseKey key;
     uint32_t sample_base;
-    int count, H, W, round_v;
+    int count, H, W, round_v;   // round_v: round v to tf32 (compact; u of the literal variant always is)
     float* v_out;               // [count][H]
 };
 
-inline size_t chain_tc_image_floats(int H) { return static_cast<size_t>(H) * (32 + 32 + 16 + 32); }
+inline size_t chain_tc_image_floats(int H, bool literal = false) {
+    return literal ? static_cast<size_t>(H) * (32 + 32 + 16 + 16 + 16) + 16 * 32 : static_cast<size_t>(H) * (32 + 32 + 16 + 32);
+}
 
-inline size_t chain_tc_smem_bytes(int H, int W) {
-    const size_t tiles = chain_tc_image_floats(H) * 4 + 2 * 128 * 128 /*Z x2*/ + 4 * 128 * 128 /*hidden chunks: 2 per slot*/;
-    const size_t floats = 3 * static_cast<size_t>(H) + static_cast<size_t>(W) * H + 16 * 16 + 16 + 16 + 32 + 16;
+inline size_t chain_tc_smem_bytes(int H, int W, bool literal = false) {
+    const size_t tiles = chain_tc_image_floats(H, literal) * 4 + 2 * 128 * 128 /*Z x2*/ + 4 * 128 * 128 /*hidden chunks: 2 per slot*/;
+    const size_t floats = literal ? 4 * static_cast<size_t>(H) + static_cast<size_t>(W) * H + 2 * 16 * 16 + 7 * 16
+                                  : 3 * static_cast<size_t>(H) + static_cast<size_t>(W) * H + 16 * 16 + 16 + 16 + 32 + 16;
     return 1024 + tiles + floats * 4 + 256;
 }
 
@@ -75,6 +91,19 @@ __device__ __forceinline__ float softplus_fast(float x) {          // ln(1 + e^x
     return x > 15.0f ? x : 0.6931471805599453f * __log2f(1.0f + e);
 }
 
+__device__ __forceinline__ float sigmoid_fast(float x) {
+    float e, r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x * -1.4426950408889634f));
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(e + 1.0f));
+    return r;
+}
+
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
 // One of the two tiles a CTA has in flight: its shared-memory operands, TMEM columns and barriers,
 // and how many times each barrier has completed (both roles count the same sequence).
 struct ChainSlot {
@@ -86,6 +115,7 @@ struct ChainSlot {
     int tile;                // current tile, -1 if the slot is idle
 };
 
+template <bool LITERAL>
 __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) {
     extern __shared__ uint8_t smem_raw[];
     const int H = a.H, W = a.W;
@@ -93,22 +123,30 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     const uint32_t base = (raw + 1023u) & ~1023u;
     uint8_t* gen = smem_raw + (base - raw);
     // weight operand tiles
-    const uint32_t t_zw1 = base;
-    const uint32_t t_w3 = t_zw1 + H * 128;
-    const uint32_t t_wmu = t_w3 + H * 128;
-    const uint32_t t_w2 = t_wmu + H * 64;
-    const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u;
+    const uint32_t t_in0 = base;                                  // [Wz | W1]   or [Wz | Wg1]
+    const uint32_t t_in1 = t_in0 + H * 128;                       // W3          or [Wh1 | Wi1]
+    const uint32_t t_wmu = t_in1 + H * 128;
+    const uint32_t t_out1 = t_wmu + H * 64;                       // W2 (32 rows per K block) or Wg2 (16 rows)
+    const uint32_t t_out2 = t_out1 + H * 64;                      // literal: Wh2
+    const uint32_t t_ws = t_out2 + H * 64;                        // literal: Ws, 16 rows x 128 bytes
+    const uint32_t image_bytes = static_cast<uint32_t>(H) * 448u + (LITERAL ? 2048u : 0u);
     const uint32_t t_act = base + image_bytes;                    // Z0, Z1, then 4 hidden-chunk buffers: 6 x 16 KB
     // fp32 side tables
     float* sbzs = reinterpret_cast<float*>(gen + image_bytes + 6 * 16384);    // bz
     float* sb1 = sbzs + H;
     float* sb3 = sb1 + H;
-    float* slr = sb3 + H;                    // [W][H]  (h_left + h_right) / 3
+    float* sbi1 = sb3 + H;                   // literal only
+    float* slr = sb3 + (LITERAL ? 2 : 1) * H;        // [W][H]  (h_left + h_right) / 3
     float* sWsig = slr + W * H;              // [16][16]
-    float* sbmu = sWsig + 256;
+    float* sWl = sWsig + 256;                // [16][16], literal only
+    float* sbmu = sWsig + (LITERAL ? 512 : 256);
     float* sbsig = sbmu + 16;
-    float* sb2 = sbsig + 16;                 // [32]
-    float* sz0 = sb2 + 32;                   // [16]
+    float* sb2 = sbsig + 16;                 // compact: [32]
+    float* sbg2 = sbsig + 16;                // literal: bg2, bh2, bl, bs, 16 each
+    float* sbh2 = sbg2 + 16;
+    float* sbl = sbh2 + 16;
+    float* sbs = sbl + 16;
+    float* sz0 = LITERAL ? sbs + 16 : sb2 + 32;      // [16]
     const uint32_t bars = smem_u32(sz0 + 16);                     // 2 slots x 7 barriers, then the drain barrier
     const uint32_t bar_drain = bars + 2 * 56;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sz0 + 16 + 32);
@@ -125,20 +163,30 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
             sbzs[i] = a.bz[i];
             sb1[i] = a.b1[i];
             sb3[i] = a.b3[i];
+            if (LITERAL) sbi1[i] = a.bi1[i];
         }
         for (int i = threadIdx.x; i < W * H; i += kChainTcThreads) slr[i] = (a.hlr[i] + a.hlr[W * H + i]) * (1.0f / 3.0f);
-        for (int i = threadIdx.x; i < 256; i += kChainTcThreads) sWsig[i] = a.Wsig[i];
+        for (int i = threadIdx.x; i < 256; i += kChainTcThreads) {
+            sWsig[i] = a.Wsig[i];
+            if (LITERAL) sWl[i] = a.Wl[i];
+        }
         if (threadIdx.x < 16) {
             sbmu[threadIdx.x] = a.bmu[threadIdx.x];
             sbsig[threadIdx.x] = a.bsig[threadIdx.x];
             sz0[threadIdx.x] = a.z0[threadIdx.x];
+            if (LITERAL) {
+                sbg2[threadIdx.x] = a.bg2[threadIdx.x];
+                sbh2[threadIdx.x] = a.bh2[threadIdx.x];
+                sbl[threadIdx.x] = a.bl[threadIdx.x];
+                sbs[threadIdx.x] = a.bs[threadIdx.x];
+            }
         }
-        if (threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
+        if (!LITERAL && threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
     }
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < 2; ++s) {
             const uint32_t b0 = bars + 56 * s;
-            mbar_init(b0, kChainEpiWarps);           // z ready
+            mbar_init(b0, kChainEpiWarps);           // latent tile (or relu(G)) ready
             mbar_init(b0 + 8, 1);                    // hidden pre-activations ready
             mbar_init(b0 + 16, kChainEpiWarps);      // hidden chunk buffer 0 written
             mbar_init(b0 + 24, kChainEpiWarps);      // hidden chunk buffer 1 written
@@ -174,9 +222,11 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         slot[s].tile = -1;
     }
     const int n_tiles = ceil_div(a.count, 128);
-    const int n_phases = W + 2;                                   // W guide steps, transition, emission hidden layer
-    // The second result of a tile (mu: 16 columns, mean | logvar: 32 columns) reuses the first columns of the
-    // tile's pre-activation block: those are multiplied only after every warp has read chunk 0.
+    // phases: W guide steps, then transition and emission hidden layer -- or gate, proposal (+ scale), first emission layer
+    const int n_phases = LITERAL ? W + 3 : W + 2;
+    const int ph_last = n_phases - 1;                             // its hidden layer goes to global memory, no second GEMM
+    // The second result of a tile (16 columns; mean | logvar: 32) reuses the first columns of the tile's
+    // pre-activation block: those are multiplied only after every warp has read chunk 0.
 
     // A hidden layer goes to the second GEMM in chunks of 64 units (two K blocks).  Each slot has one chunk buffer
     // (its two 16 KB tiles); the chunks of the two tiles in flight are produced alternately -- (chunk 0, slot 0),
@@ -187,7 +237,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
 
     if (warp == 0) {
         // ---------------- MMA issuer -------------------------------------------------------------------
-        const uint32_t idesc_h = instr_desc_tf32(H), idesc_mu = instr_desc_tf32(16), idesc_head = instr_desc_tf32(32);
+        const uint32_t idesc_h = instr_desc_tf32(H), idesc_16 = instr_desc_tf32(16), idesc_head = instr_desc_tf32(32);
         bool ok = true;
         for (int t0 = blockIdx.x; ok && t0 < n_tiles; t0 += 2 * gridDim.x) {
             slot[0].tile = t0;
@@ -202,7 +252,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                     ++sl.nz;
                     tc_fence_after();
                     if (lane == 0) {
-                        const uint32_t b_tile = ph < W ? t_zw1 : (ph == W ? t_zw1 + 64u : t_w3);
+                        const uint32_t b_tile = ph < W ? t_in0 : (ph == W ? t_in0 + 64u : (ph == W + 1 ? t_in1 : t_in1 + 64u));
                         const uint64_t a_desc = make_smem_desc(sl.t_z), b_desc = make_smem_desc(b_tile);
                         umma_tf32(sl.tmem, a_desc, b_desc, idesc_h, 0u);
                         umma_tf32(sl.tmem, a_desc + 2, b_desc + 2, idesc_h, 1u);
@@ -210,10 +260,10 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                     }
                     __syncwarp();
                 }
-                if (ph > W) continue;                              // the emission hidden layer has no second GEMM here
-                const uint32_t b_base = ph < W ? t_wmu : t_w2;
-                const uint32_t slab = ph < W ? 16u * 128u : 32u * 128u;
-                const uint32_t idesc2 = ph < W ? idesc_mu : idesc_head;
+                if (ph == ph_last) continue;                       // the last hidden layer has no second GEMM here
+                const uint32_t b_base = ph < W ? t_wmu : (ph == W ? t_out1 : t_out2);
+                const uint32_t slab = LITERAL || ph < W ? 16u * 128u : 32u * 128u;
+                const uint32_t idesc2 = LITERAL || ph < W ? idesc_16 : idesc_head;
                 for (int c = 0; ok && c < n_chunks64; ++c) {        // second GEMM, chunk by chunk as the epilogue delivers
 #pragma unroll
                     for (int s = 0; s < 2; ++s) {
@@ -238,6 +288,23 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                         __syncwarp();
                     }
                 }
+                if (!LITERAL || ph != W + 1) continue;
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {                       // scale: Ws relu(G), relu(G) sits in the latent tile
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    ok = mbar_wait(sl.bar_z, sl.nz & 1u, abort_flag, a.st);
+                    if (!ok) continue;
+                    ++sl.nz;
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint64_t a_desc = make_smem_desc(sl.t_z), b_desc = make_smem_desc(t_ws);
+                        umma_tf32(sl.tmem, a_desc, b_desc, idesc_16, 0u);
+                        umma_tf32(sl.tmem, a_desc + 2, b_desc + 2, idesc_16, 1u);
+                        umma_commit(sl.bar_acc2);
+                    }
+                    __syncwarp();
+                }
             }
         }
         if (!ok) {
@@ -254,6 +321,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         const uint32_t step = a.st->step;
         const uint32_t hb_off = static_cast<uint32_t>(cg >> 1) * 16384u;          // K block of the chunk this warp writes
         const int hb_chunk = 4 * (cg & 1);                                        // its first 16-byte chunk in a row
+        float gate_own[2][4], lin_own[2][4], G_own[2][4];     // literal: per tile in flight, latent dimensions 4cg..4cg+3
         bool ok = true;
         for (int t0 = blockIdx.x; ok && t0 < n_tiles; t0 += 2 * gridDim.x) {
             slot[0].tile = t0;
@@ -269,7 +337,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                 if (lane == 0) mbar_arrive(slot[s].bar_z);
             }
             for (int ph = 0; ok && ph < n_phases; ++ph) {
-                const float* bias = ph < W ? sbzs : (ph == W ? sb1 : sb3);
+                const float* bias = ph < W ? sbzs : (ph == W ? sb1 : (ph == W + 1 ? sb3 : sbi1));
                 const float* lr = slr + (ph < W ? ph : 0) * H;
                 // ---- hidden layer of both tiles: bias, activation, next A operand (or v) -----------------
                 for (int c = 0; ok && c < n_chunks64; ++c) {
@@ -301,12 +369,15 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                                     asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(__uint_as_float(acc[4 * g + i]) + bv[i]));
                                     h[4 * g + i] = fmaf(t, 1.0f / 3.0f, lv[i]);
                                 }
+                            } else if (LITERAL && ph == ph_last) {  // u = Wi1 z' + bi1: no activation
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) h[4 * g + i] = __uint_as_float(acc[4 * g + i]) + bv[i];
                             } else {
 #pragma unroll
                                 for (int i = 0; i < 4; ++i) h[4 * g + i] = fmaxf(__uint_as_float(acc[4 * g + i]) + bv[i], 0.0f);
                             }
                         }
-                        if (ph <= W) {
+                        if (ph != ph_last) {
                             if (sl.nu >= 1) {                      // the buffer's previous contents must have been multiplied
                                 ok = mbar_wait(sl.bar_hfree, (sl.nu - 1u) & 1u, abort_flag, a.st);
                                 if (!ok) continue;
@@ -324,7 +395,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                         } else {
                             const int k = sl.tile * 128 + row;
                             if (k < a.count) {
-                                if (a.round_v) {
+                                if (LITERAL || a.round_v) {
 #pragma unroll
                                     for (int i = 0; i < 16; ++i) h[i] = tf32_rna(h[i]);
                                 }
@@ -334,22 +405,25 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                         }
                     }
                 }
-                if (!ok || ph > W) continue;
-                // ---- second result of both tiles: the next latent -----------------------------------------
+                if (!ok || ph == ph_last) continue;
+                // ---- second result of both tiles: the next latent (literal: gate, then G and relu(G)) ------------
 #pragma unroll
                 for (int s = 0; s < 2; ++s) {
                     ChainSlot& sl = slot[s];
                     if (!ok || sl.tile < 0) continue;
                     const uint32_t sample = a.sample_base + static_cast<uint32_t>(sl.tile * 128 + row);
                     float eps[4];                                   // drawn before the wait: the noise does not depend on the result
-                    normal4_fast(static_cast<uint32_t>(cg), sample, ph < W ? static_cast<uint32_t>(ph) : kStreamTransition, step,
-                                 a.key.seed_lo, a.key.seed_hi, eps);
+                    if (!LITERAL || ph < W)
+                        normal4_fast(static_cast<uint32_t>(cg), sample, ph < W ? static_cast<uint32_t>(ph) : kStreamTransition, step,
+                                     a.key.seed_lo, a.key.seed_hi, eps);
                     ok = mbar_wait(sl.bar_acc2, sl.na & 1u, abort_flag, a.st);
                     if (!ok) continue;
                     ++sl.na;
                     tc_fence_after();
                     float z_own[4];
+                    bool store_z = true;
                     if (ph < W) {
+                        // guide: z = mu + softplus(Wsig mu + bsig) * eps
                         uint32_t mu_bits[16];
                         tmem_ld16(sl.tmem + lane_off, mu_bits);
                         tmem_ld_wait();
@@ -368,7 +442,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                                 if (gg == cg) own = mu[4 * gg + c];
                             z_own[c] = fmaf(softplus_fast(pre), eps[c], own);
                         }
-                    } else {
+                    } else if constexpr (!LITERAL) {
                         uint32_t mean_bits[16], lv_bits[16];
                         tmem_ld16(sl.tmem + lane_off, mean_bits);
                         tmem_ld16(sl.tmem + lane_off + 16, lv_bits);
@@ -381,6 +455,77 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
                                 if (gg == cg) { mean = __uint_as_float(mean_bits[4 * gg + c]); lv = __uint_as_float(lv_bits[4 * gg + c]); }
                             z_own[c] = fmaf(exp_half_fast(lv + sb2[16 + 4 * cg + c]), eps[c], mean + sb2[4 * cg + c]);
                         }
+                    } else {
+                        uint32_t res_bits[16];
+                        tmem_ld16(sl.tmem + lane_off, res_bits);
+                        tmem_ld_wait();
+                        float own[4];                               // this thread's four of the 16 results
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            own[c] = 0.0f;
+#pragma unroll
+                            for (int gg = 0; gg < 4; ++gg)
+                                if (gg == cg) own[c] = __uint_as_float(res_bits[4 * gg + c]);
+                        }
+                        if (ph == W) {
+                            // gate g, and the linear map Wl z + bl from the latent tile (it stays as it is for the proposal)
+                            float z[16];
+#pragma unroll
+                            for (int e4 = 0; e4 < 4; ++e4) {
+                                const float4 zq = ld_shared_v4(sl.t_z + sw128(row, e4));
+                                z[4 * e4 + 0] = zq.x; z[4 * e4 + 1] = zq.y; z[4 * e4 + 2] = zq.z; z[4 * e4 + 3] = zq.w;
+                            }
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                gate_own[s][c] = sigmoid_fast(own[c] + sbg2[4 * cg + c]);
+                                const float* wrow = sWl + (4 * cg + c) * 16;
+                                float lin = sbl[4 * cg + c];
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) lin = fmaf(wrow[e], z[e], lin);
+                                lin_own[s][c] = lin;
+                            }
+                            store_z = false;
+                        } else {
+                            // proposal h -> G = (1 - g) * lin + g * h; relu(G) replaces the latent tile for the scale product
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) {
+                                const float prop = own[c] + sbh2[4 * cg + c];
+                                G_own[s][c] = fmaf(gate_own[s][c], prop - lin_own[s][c], lin_own[s][c]);
+                                z_own[c] = fmaxf(G_own[s][c], 0.0f);
+                            }
+                        }
+                    }
+                    if (store_z) {
+                        st_shared_v4(sl.t_z + sw128(row, cg), tf32_rna(z_own[0]), tf32_rna(z_own[1]), tf32_rna(z_own[2]), tf32_rna(z_own[3]));
+                        fence_proxy_async();
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(sl.bar_z);
+                }
+                if (!LITERAL || !ok || ph != W + 1) continue;
+                // ---- literal: scale of both tiles, z' = G + softplus(Ws relu(G) + bs) * eps ------------------
+#pragma unroll
+                for (int s = 0; s < 2; ++s) {
+                    ChainSlot& sl = slot[s];
+                    if (!ok || sl.tile < 0) continue;
+                    const uint32_t sample = a.sample_base + static_cast<uint32_t>(sl.tile * 128 + row);
+                    float eps[4], z_own[4];
+                    normal4_fast(static_cast<uint32_t>(cg), sample, kStreamTransition, step, a.key.seed_lo, a.key.seed_hi, eps);
+                    ok = mbar_wait(sl.bar_acc2, sl.na & 1u, abort_flag, a.st);
+                    if (!ok) continue;
+                    ++sl.na;
+                    tc_fence_after();
+                    uint32_t res_bits[16];
+                    tmem_ld16(sl.tmem + lane_off, res_bits);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float pre = 0.0f;
+#pragma unroll
+                        for (int gg = 0; gg < 4; ++gg)
+                            if (gg == cg) pre = __uint_as_float(res_bits[4 * gg + c]);
+                        z_own[c] = fmaf(softplus_fast(pre + sbs[4 * cg + c]), eps[c], G_own[s][c]);
                     }
                     st_shared_v4(sl.t_z + sw128(row, cg), tf32_rna(z_own[0]), tf32_rna(z_own[1]), tf32_rna(z_own[2]), tf32_rna(z_own[3]));
                     fence_proxy_async();

@@ -16,7 +16,7 @@
 // second results (mu: 32 columns; mean | logvar: 64 columns) reuse columns [0, 64), which is why the
 // first two chunks of a phase are produced before the first of them is multiplied.
 //
-// LITERAL = true runs the networks as Section 3.1.3 prints them (see chain_tc_literal.cuh for the formulas) on the
+// LITERAL = true runs the networks as Section 3.1.3 prints them (see chain_tc.cuh for the formulas) on the
 // same skeleton: after the guide steps come the gate (Wg1, Wg2), the proposal (Wh1, Wh2; its result is combined
 // with the gate and the linear map Wl z + bl, which the epilogue threads compute from the latent tile, into G;
 // relu(G) then takes the latent tile's place for one more small product with Ws, which stays resident), and the
@@ -24,7 +24,6 @@
 // proposal A = Wh1, B = Wh2; emission A = Wi1.
 #pragma once
 #include "chain_tc.cuh"
-#include "chain_tc_literal.cuh"      // sigmoid_fast, ld_shared_v4
 
 namespace cutoff {
 namespace tc {

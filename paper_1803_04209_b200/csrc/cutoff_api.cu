@@ -17,7 +17,6 @@
 #include "chain_tc32.cuh"
 #include "kernels_literal.cuh"
 #include "gemm_tc.cuh"
-#include "chain_tc_literal.cuh"
 #include "pipe_rates.cuh"
 #include "kernels_eval.cuh"
 #include "fit_api.cuh"
@@ -289,16 +288,22 @@ void launch_chain_t(cutoff_ctx* c, uint32_t sample_base, int count, size_t smem)
 }
 
 void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
-    tc::ChainTcArgs a;
+    tc::ChainTcArgs a{};
     const ModelDev& m = c->m;
     a.image = c->d_chain_image;
     a.bz = m.bz; a.b1 = m.b1; a.b3 = m.b3; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig; a.b2 = m.b2; a.z0 = m.z0;
+    if (c->chain_tcl) {
+        const LiteralDev& l = c->lit;
+        a.b1 = l.bg1; a.b3 = l.bh1; a.b2 = nullptr;
+        a.bi1 = l.bi1; a.bg2 = l.bg2; a.bh2 = l.bh2; a.Wl = l.Wl; a.bl = l.bl; a.bs = l.bs;
+    }
     a.hlr = c->d_hlr; a.st = c->d_state;
     a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
     a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.round_v = 1; a.v_out = c->d_v;
     const int tiles = ceil_div(count, 128);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    tc::k_chain_tc<<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W), c->stream>>>(a);
+    if (c->chain_tcl) tc::k_chain_tc<true><<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W, true), c->stream>>>(a);
+    else tc::k_chain_tc<false><<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W), c->stream>>>(a);
     c->launches += 1;
 }
 
@@ -330,24 +335,8 @@ void launch_chain_literal_t(cutoff_ctx* c, uint32_t sample_base, int count) {
         c->m, c->lit, c->d_hlr, c->d_state, key, sample_base, count, c->use_tc ? 1 : 0, c->d_v);
 }
 
-void launch_chain_tc_literal(cutoff_ctx* c, uint32_t sample_base, int count) {
-    tc::ChainTclArgs a;
-    const ModelDev& m = c->m;
-    const LiteralDev& l = c->lit;
-    a.image = c->d_chain_image;
-    a.bz = m.bz; a.bg1 = l.bg1; a.bh1 = l.bh1; a.bi1 = l.bi1; a.bmu = m.bmu; a.bsig = m.bsig; a.Wsig = m.Wsig;
-    a.bg2 = l.bg2; a.bh2 = l.bh2; a.Wl = l.Wl; a.bl = l.bl; a.bs = l.bs; a.z0 = m.z0;
-    a.hlr = c->d_hlr; a.st = c->d_state;
-    a.key = NoiseKey{static_cast<uint32_t>(c->cfg.seed), static_cast<uint32_t>(c->cfg.seed >> 32)};
-    a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.u_out = c->d_v;
-    const int tiles = ceil_div(count, 128);
-    const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    tc::k_chain_tc_literal<<<grid, tc::kChainTcThreads, tc::chain_tcl_smem_bytes(c->H, c->W), c->stream>>>(a);
-    c->launches += 1;
-}
-
 void launch_chain(cutoff_ctx* c, uint32_t sample_base, int count) {
-    if (c->chain_tcl) { launch_chain_tc_literal(c, sample_base, count); return; }
+    if (c->chain_tcl) { launch_chain_tc(c, sample_base, count); return; }
     if (c->chain_tcl32) { launch_chain_tc32(c, sample_base, count); return; }
     if (c->literal) {
         switch (c->D) {
@@ -631,10 +620,10 @@ cudaError_t set_kernel_attributes(const cutoff_ctx* c) {
     if (e == cudaSuccess) e = allow_smem(tc::k_emit_tc2, tc::kSmem2Bytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_gemm_relu_tc, tc::kSmemBytes);
     if (e == cudaSuccess) e = allow_smem(tc::k_emit_dual_tc, tc::kDualSmemBytes);
-    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc<false>, 227 * 1024);
+    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc<true>, 227 * 1024);
     if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32<false>, 227 * 1024);
     if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc32<true>, 227 * 1024);
-    if (e == cudaSuccess) e = allow_smem(tc::k_chain_tc_literal, 227 * 1024);
     return e;
 }
 
@@ -718,7 +707,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     c->chain_tc = !c->literal && c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
                   tc::chain_tc_smem_bytes(c->H, c->W) <= 227 * 1024;
     c->chain_tcl = c->literal && c->use_tc && c->D == tc::kChainD && c->H % 64 == 0 && c->H <= 256 &&
-                   tc::chain_tcl_smem_bytes(c->H, c->W) <= 227 * 1024;
+                   tc::chain_tc_smem_bytes(c->H, c->W, true) <= 227 * 1024;
     c->chain_tc32 = !c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
                     (c->H <= 256 || (c->H - 256) % 16 == 0) && tc::chain_tc32_smem_bytes(c->H, c->W) <= 227 * 1024;
     c->chain_tcl32 = c->literal && c->use_tc && c->D == tc::kChain32D && c->H % 32 == 0 && c->H <= 512 &&
@@ -743,7 +732,7 @@ int cutoff_create(cutoff_ctx** out, const cutoff_config* cfg) {
     CREATE_CHECK(cudaMalloc(&c->d_WhR, sizeof(float) * 2 * c->H * c->H));
     if (c->chain_tc) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H)));
     if (c->chain_tc32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H)));
-    if (c->chain_tcl) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tcl_image_floats(c->H)));
+    if (c->chain_tcl) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc_image_floats(c->H, true)));
     if (c->chain_tcl32) CREATE_CHECK(cudaMalloc(&c->d_chain_image, sizeof(float) * tc::chain_tc32_image_floats(c->H, true)));
     CREATE_CHECK(cudaMalloc(&c->d_ring, sizeof(float) * c->W * c->N));
     CREATE_CHECK(cudaMalloc(&c->d_stage, sizeof(float) * c->N));
@@ -908,7 +897,7 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     if (c->chain_tcl) {
         // Literal variant, D = 16: [Wz | Wg1] and [Wh1 | Wi1] as [H rows][32], Wmu, Wg2, Wh2 as H/32 K blocks of
         // [16 rows][32], Ws as [16 rows][32] (columns 16.. zero), all tf32 in the swizzled shared-memory layout.
-        std::vector<float> img(tc::chain_tcl_image_floats(c->H), 0.0f);
+        std::vector<float> img(tc::chain_tc_image_floats(c->H, true), 0.0f);
         const float* wz = host.data() + off[8];      // [H][D]
         const float* wg1 = host.data() + off[15];
         const float* wh1 = host.data() + off[19];
