@@ -191,6 +191,21 @@ size_t swz(size_t row, size_t col) {
     return (row >> 3) * 256 + (row & 7) * 32 + ((((col >> 2) ^ (row & 7)) << 2) | (col & 3));
 }
 
+// A first-layer matrix w [rows][cols] (cols <= 32) into columns col0 .. col0 + cols - 1 of a swizzled tile of
+// `rows` rows x 32, rounded to tf32: the B operand of hidden = act(W z + b), K = the latent size.
+void put_first_layer(float* tile, const float* w, size_t rows, size_t cols, size_t col0) {
+    for (size_t n = 0; n < rows; ++n)
+        for (size_t k = 0; k < cols; ++k) tile[swz(n, col0 + k)] = host_tf32(w[n * cols + k]);
+}
+
+// A second-layer matrix w [out_rows][H] as H / 32 K blocks of `block_rows` rows x 32 (out_rows <= block_rows; the
+// other rows stay as they are), swizzled and rounded to tf32: the B operand of out = W hidden, K = H.
+void put_second_layer(float* tiles, const float* w, size_t out_rows, size_t H, size_t block_rows) {
+    for (size_t kb = 0; kb < H / 32; ++kb)
+        for (size_t o = 0; o < out_rows; ++o)
+            for (size_t jj = 0; jj < 32; ++jj) tiles[kb * block_rows * 32 + swz(o, jj)] = host_tf32(w[o * H + kb * 32 + jj]);
+}
+
 int next_pow2(int n) {
     int p = 1;
     while (p < n) p <<= 1;
@@ -867,108 +882,60 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
         }
         CU_CHECK(c, cudaMemcpy(c->d_WhR, whr.data(), whr.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
-    if (c->chain_tc) {
-        // Operand tiles of the tensor-core chain as they will sit in shared memory: tf32 (nearest, ties
-        // away), K-major rows of 32 values, 16-byte chunks XOR-swizzled with the row index modulo 8.
-        std::vector<float> img(tc::chain_tc_image_floats(c->H), 0.0f);
-        const float* wz = host.data() + off[8];      // [H][D]
-        const float* w1 = host.data() + off[15];     // [H][D]
-        const float* w3 = host.data() + off[19];     // [H][D]
-        const float* wmu = host.data() + off[10];    // [D][H]
-        const float* w2 = host.data() + off[17];     // [2D][H]
-        float* t_zw1 = img.data();
-        float* t_w3 = t_zw1 + H * 32;
-        float* t_wmu = t_w3 + H * 32;
-        float* t_w2 = t_wmu + H * 16;
-        for (size_t n = 0; n < H; ++n)
-            for (size_t k = 0; k < D; ++k) {
-                t_zw1[swz(n, k)] = host_tf32(wz[n * D + k]);
-                t_zw1[swz(n, 16 + k)] = host_tf32(w1[n * D + k]);
-                t_w3[swz(n, k)] = host_tf32(w3[n * D + k]);
-            }
-        for (size_t kb = 0; kb < H / 32; ++kb)
-            for (size_t jj = 0; jj < 32; ++jj) {
-                for (size_t d = 0; d < D; ++d) t_wmu[kb * 16 * 32 + swz(d, jj)] = host_tf32(wmu[d * H + kb * 32 + jj]);
-                for (size_t o = 0; o < 2 * D; ++o) t_w2[kb * 32 * 32 + swz(o, jj)] = host_tf32(w2[o * H + kb * 32 + jj]);
-            }
-        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
-    }
-
-    if (c->chain_tcl) {
-        // Literal variant, D = 16: [Wz | Wg1] and [Wh1 | Wi1] as [H rows][32], Wmu, Wg2, Wh2 as H/32 K blocks of
-        // [16 rows][32], Ws as [16 rows][32] (columns 16.. zero), all tf32 in the swizzled shared-memory layout.
-        std::vector<float> img(tc::chain_tc_image_floats(c->H, true), 0.0f);
-        const float* wz = host.data() + off[8];      // [H][D]
-        const float* wg1 = host.data() + off[15];
-        const float* wh1 = host.data() + off[19];
-        const float* wi1 = host.data() + off[27];
-        const float* second[3] = {host.data() + off[10], host.data() + off[17], host.data() + off[21]};   // Wmu, Wg2, Wh2: [D][H]
-        const float* ws = host.data() + off[25];     // [D][D]
-        float* t_zg = img.data();
-        float* t_hi = t_zg + H * 32;
-        float* t_second = t_hi + H * 32;             // three tiles of H x 16 floats
-        float* t_ws = t_second + 3 * H * 16;
-        for (size_t n = 0; n < H; ++n)
-            for (size_t k = 0; k < D; ++k) {
-                t_zg[swz(n, k)] = host_tf32(wz[n * D + k]);
-                t_zg[swz(n, 16 + k)] = host_tf32(wg1[n * D + k]);
-                t_hi[swz(n, k)] = host_tf32(wh1[n * D + k]);
-                t_hi[swz(n, 16 + k)] = host_tf32(wi1[n * D + k]);
-            }
-        for (int t = 0; t < 3; ++t)
-            for (size_t kb = 0; kb < H / 32; ++kb)
-                for (size_t jj = 0; jj < 32; ++jj)
-                    for (size_t d = 0; d < D; ++d)
-                        t_second[t * H * 16 + kb * 16 * 32 + swz(d, jj)] = host_tf32(second[t][d * H + kb * 32 + jj]);
-        for (size_t o = 0; o < D; ++o)
-            for (size_t e = 0; e < D; ++e) t_ws[swz(o, e)] = host_tf32(ws[o * D + e]);
-        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
-    }
-
-    if (c->chain_tc32) {
-        // D = 32: six tiles of H x 32 tf32 values each -- Wz, W1, W3 as [H rows][32], Wmu and the two halves of W2 as
-        // H/32 K blocks of [32 rows][32] -- in the swizzled shared-memory layout, staged by the kernel phase by phase
+    // Operand tiles of the tensor-core chain kernels as they will sit in shared memory: tf32 (nearest, ties away),
+    // K-major rows of 32 values, 16-byte chunks XOR-swizzled with the row index modulo 8.
+    if (c->chain_tc || c->chain_tcl || c->chain_tc32 || c->chain_tcl32) {
+        const bool lit = c->chain_tcl || c->chain_tcl32;
+        const float* wz = host.data() + off[8];                  // first layers, [H][D]: Wz; W1 or Wg1; W3 or Wh1; Wi1
+        const float* wa = host.data() + off[15];
+        const float* wb = host.data() + off[19];
+        const float* wi1 = lit ? host.data() + off[27] : nullptr;
+        const float* wmu = host.data() + off[10];                // second layers, [D][H] ([2D][H] for W2): Wmu; W2 or Wg2; Wh2
+        const float* wc = host.data() + off[17];
+        const float* wh2 = lit ? host.data() + off[21] : nullptr;
+        const float* ws = lit ? host.data() + off[25] : nullptr; // [D][D]
         const size_t tile = H * 32;
-        std::vector<float> img(tc::chain_tc32_image_floats(c->H), 0.0f);
-        const float* wz = host.data() + off[8];
-        const float* w1 = host.data() + off[15];
-        const float* w3 = host.data() + off[19];
-        const float* wmu = host.data() + off[10];    // [32][H]
-        const float* w2 = host.data() + off[17];     // [64][H]: rows 0..31 mean, 32..63 log-variance
-        for (size_t n = 0; n < H; ++n)
-            for (size_t k = 0; k < 32; ++k) {
-                img[0 * tile + swz(n, k)] = host_tf32(wz[n * 32 + k]);
-                img[1 * tile + swz(n, k)] = host_tf32(w1[n * 32 + k]);
-                img[2 * tile + swz(n, k)] = host_tf32(w3[n * 32 + k]);
+        std::vector<float> img;
+        if (c->chain_tc || c->chain_tcl) {
+            // D = 16: two first-layer matrices share a tile (columns 0..15 and 16..31); second-layer K blocks of 16 rows
+            // (W2: 32).  compact: [Wz|W1], W3, Wmu, W2;  literal: [Wz|Wg1], [Wh1|Wi1], Wmu, Wg2, Wh2, Ws (16 rows)
+            img.assign(tc::chain_tc_image_floats(c->H, lit), 0.0f);
+            float* t_in0 = img.data();
+            float* t_in1 = t_in0 + tile;
+            float* t_wmu = t_in1 + tile;
+            float* t_out1 = t_wmu + H * 16;
+            put_first_layer(t_in0, wz, H, D, 0);
+            put_first_layer(t_in0, wa, H, D, 16);
+            put_first_layer(t_in1, wb, H, D, 0);
+            put_second_layer(t_wmu, wmu, D, H, 16);
+            if (lit) {
+                float* t_out2 = t_out1 + H * 16;
+                put_first_layer(t_in1, wi1, H, D, 16);
+                put_second_layer(t_out1, wc, D, H, 16);
+                put_second_layer(t_out2, wh2, D, H, 16);
+                put_first_layer(t_out2 + H * 16, ws, D, D, 0);
+            } else {
+                put_second_layer(t_out1, wc, 2 * D, H, 32);
             }
-        for (size_t kb = 0; kb < H / 32; ++kb)
-            for (size_t jj = 0; jj < 32; ++jj)
-                for (size_t d = 0; d < 32; ++d) {
-                    img[3 * tile + kb * 1024 + swz(d, jj)] = host_tf32(wmu[d * H + kb * 32 + jj]);
-                    img[4 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[d * H + kb * 32 + jj]);
-                    img[5 * tile + kb * 1024 + swz(d, jj)] = host_tf32(w2[(32 + d) * H + kb * 32 + jj]);
-                }
-        CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
-    }
-
-    if (c->chain_tcl32) {
-        // Literal variant, D = 32: Wz, Wg1, Wh1, Wi1 as [H rows][32]; Wmu, Wg2, Wh2 as H/32 K blocks of [32 rows][32];
-        // Ws as [32 rows][32]; all tf32 in the swizzled shared-memory layout, staged by the kernel phase by phase.
-        const size_t tile = H * 32;
-        std::vector<float> img(tc::chain_tc32_image_floats(c->H, true), 0.0f);
-        const float* first[4] = {host.data() + off[8], host.data() + off[15], host.data() + off[19], host.data() + off[27]};   // Wz Wg1 Wh1 Wi1: [H][32]
-        const float* second[3] = {host.data() + off[10], host.data() + off[17], host.data() + off[21]};                       // Wmu Wg2 Wh2: [32][H]
-        const float* ws = host.data() + off[25];                                                                              // [32][32]
-        for (int t = 0; t < 4; ++t)
-            for (size_t n = 0; n < H; ++n)
-                for (size_t k = 0; k < 32; ++k) img[t * tile + swz(n, k)] = host_tf32(first[t][n * 32 + k]);
-        for (int t = 0; t < 3; ++t)
-            for (size_t kb = 0; kb < H / 32; ++kb)
-                for (size_t jj = 0; jj < 32; ++jj)
-                    for (size_t d = 0; d < 32; ++d)
-                        img[(4 + t) * tile + kb * 1024 + swz(d, jj)] = host_tf32(second[t][d * H + kb * 32 + jj]);
-        for (size_t o = 0; o < 32; ++o)
-            for (size_t e = 0; e < 32; ++e) img[7 * tile + swz(o, e)] = host_tf32(ws[o * 32 + e]);
+        } else {
+            // D = 32: every matrix has a tile of H x 32 of its own, staged by the kernel phase by phase.
+            // compact: Wz, W1, W3, Wmu, W2 mean rows, W2 log-variance rows;  literal: Wz, Wg1, Wh1, Wi1, Wmu, Wg2, Wh2, Ws
+            img.assign(tc::chain_tc32_image_floats(c->H, lit), 0.0f);
+            put_first_layer(img.data() + 0 * tile, wz, H, 32, 0);
+            put_first_layer(img.data() + 1 * tile, wa, H, 32, 0);
+            put_first_layer(img.data() + 2 * tile, wb, H, 32, 0);
+            if (lit) {
+                put_first_layer(img.data() + 3 * tile, wi1, H, 32, 0);
+                put_second_layer(img.data() + 4 * tile, wmu, 32, H, 32);
+                put_second_layer(img.data() + 5 * tile, wc, 32, H, 32);
+                put_second_layer(img.data() + 6 * tile, wh2, 32, H, 32);
+                put_first_layer(img.data() + 7 * tile, ws, 32, 32, 0);
+            } else {
+                put_second_layer(img.data() + 3 * tile, wmu, 32, H, 32);
+                put_second_layer(img.data() + 4 * tile, wc, 32, H, 32);
+                put_second_layer(img.data() + 5 * tile, wc + 32 * H, 32, H, 32);
+            }
+        }
         CU_CHECK(c, cudaMemcpy(c->d_chain_image, img.data(), img.size() * sizeof(float), cudaMemcpyHostToDevice));
     }
 
