@@ -598,16 +598,16 @@ def main():
     # few MB that every SM re-reads, hidden vectors from one of tens of MB.
     if wl.precision and not literal and not args.no_measure_alu_peak:
         from paper_1803_04209_b200 import binding as _b
-        stream = _b.measure_operand_stream(local_rank)
+        op_rates = _b.measure_operand_stream(local_rank)
         n_tiles = -(-wl.S // 128) * -(-wl.N // 128)
         k_bytes = -(-wl.H // 32) * 128                               # bytes of one operand row (K blocks of 32 floats)
         bytes_w, bytes_v = n_tiles * 256 * k_bytes, n_tiles * 128 * k_bytes
-        t_stream = bytes_w / (stream["weights_2mb"] * 1e9) + bytes_v / (stream["hidden_64mb"] * 1e9)
+        t_stream = bytes_w / (op_rates["weights_2mb"] * 1e9) + bytes_v / (op_rates["hidden_64mb"] * 1e9)
         roofline["emission_stream"] = {
             "bound": "l2 -> shared memory operand stream",
             "bytes_per_launch": bytes_w + bytes_v,
             "achieved_gbs": round((bytes_w + bytes_v) / (stage_avg["emission"] * 1e-3) / 1e9, 1),
-            "peak_gbs": {k: round(v, 1) for k, v in stream.items()},
+            "peak_gbs": {k: round(v, 1) for k, v in op_rates.items()},
             "model_ms": round(t_stream * 1e3, 4),
             "frac": round(t_stream / (stage_avg["emission"] * 1e-3), 4),
             "peak_source": "measured (cutoff_measure_operand_stream, this run): the kernel's own copies, nothing consuming them",
