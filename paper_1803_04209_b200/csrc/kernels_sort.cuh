@@ -343,10 +343,15 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
         }
         const float* src = buf0 + b * ldx;
         float v[E];
+        if (N == 32 * E) {                             // a full row: no padding keys to put in
 #pragma unroll
-        for (int r = 0; r < E; ++r) {
-            const int e = r * 32 + lane;
-            v[r] = e < N ? src[e] : INFINITY;
+            for (int r = 0; r < E; ++r) v[r] = src[r * 32 + lane];
+        } else {
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const int e = r * 32 + lane;
+                v[r] = e < N ? src[e] : INFINITY;
+            }
         }
         __syncwarp();
         warp_bitonic_sort<float, E>(v, lane);
