@@ -578,7 +578,19 @@ def main():
     t_alu = minmax_ops / lane_rate("minmax") + fma_ops / lane_rate("fma")
     t_xchg = xchg_ops / lane_rate("shuffle")
     t_model = max(t_tc, t_alu, t_xchg)
+    # Stage by stage: each of the three large stages against the one unit its arithmetic runs on (tensor cores for the
+    # products that use them, the FMA rate for those that do not, the min/max rate for the sort), and their sum against
+    # the time the three take one after the other.  Looser than path_frac (it lets no stage overlap another), stricter
+    # than the dominant kernel's own fraction.
+    ideal = {
+        "chain": 2 * work["chain"][1] / tensor_peak if chain_on_tensor else work["chain"][1] / lane_rate("fma"),
+        "emission": work["emission"][1] / (tensor_peak if work["emission"][0] == "tensor" else lane_rate("fma")),
+        "sort": minmax_ops / lane_rate("minmax"),
+    }
+    big = ("chain", "emission", "sort")
     roofline.update({
+        "stage_frac": {k: round(ideal[k] / (stage_avg[k] * 1e-3), 4) for k in big},
+        "path_frac_sum": sum(ideal[k] for k in big) / (sum(stage_avg[k] for k in big) * 1e-3),
         "path_frac": t_model / (ms_per_step * 1e-3),
         "path_model_ms": {"tensor": round(t_tc * 1e3, 4), "alu": round(t_alu * 1e3, 4), "exchange": round(t_xchg * 1e3, 4)},
         "path_model_sources": {
