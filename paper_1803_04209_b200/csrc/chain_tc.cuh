@@ -149,16 +149,35 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
     float* sz0 = LITERAL ? sbs + 16 : sb2 + 32;      // [16]
     const uint32_t bars = smem_u32(sz0 + 16);                     // 2 slots x 7 barriers, then the drain barrier
     const uint32_t bar_drain = bars + 2 * 56;
+    const uint32_t bar_img = bar_drain + 8;                       // the operand image has landed
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sz0 + 16 + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sz0 + 16 + 34);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- one-time set-up: operand image, side tables, barriers, TMEM --------------------------------
+    // ---- one-time set-up: barriers, operand image (bulk copies, while the side tables are filled), TMEM ----------
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < 2; ++s) {
+            const uint32_t b0 = bars + 56 * s;
+            mbar_init(b0, kChainEpiWarps);           // latent tile (or relu(G)) ready
+            mbar_init(b0 + 8, 1);                    // hidden pre-activations ready
+            mbar_init(b0 + 16, kChainEpiWarps);      // hidden chunk buffer 0 written
+            mbar_init(b0 + 24, kChainEpiWarps);      // hidden chunk buffer 1 written
+            mbar_init(b0 + 32, 1);                   // hidden chunk buffer 0 multiplied
+            mbar_init(b0 + 40, 1);                   // hidden chunk buffer 1 multiplied
+            mbar_init(b0 + 48, 1);                   // second result ready
+        }
+        mbar_init(bar_drain, 1);
+        mbar_init(bar_img, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        mbar_arrive_expect_tx(bar_img, image_bytes);
+        for (uint32_t off = 0; off < image_bytes; off += 32768u) {
+            const uint32_t n = image_bytes - off < 32768u ? image_bytes - off : 32768u;
+            bulk_load_1d(base + off, reinterpret_cast<const uint8_t*>(a.image) + off, n, bar_img);
+        }
+    }
     {
-        const float4* src = reinterpret_cast<const float4*>(a.image);
-        float4* dst = reinterpret_cast<float4*>(gen);
-        for (uint32_t i = threadIdx.x; i < image_bytes / 16; i += kChainTcThreads) dst[i] = src[i];
         for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
             sbzs[i] = a.bz[i];
             sb1[i] = a.b1[i];
@@ -183,31 +202,17 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         }
         if (!LITERAL && threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
     }
-    if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < 2; ++s) {
-            const uint32_t b0 = bars + 56 * s;
-            mbar_init(b0, kChainEpiWarps);           // latent tile (or relu(G)) ready
-            mbar_init(b0 + 8, 1);                    // hidden pre-activations ready
-            mbar_init(b0 + 16, kChainEpiWarps);      // hidden chunk buffer 0 written
-            mbar_init(b0 + 24, kChainEpiWarps);      // hidden chunk buffer 1 written
-            mbar_init(b0 + 32, 1);                   // hidden chunk buffer 0 multiplied
-            mbar_init(b0 + 40, 1);                   // hidden chunk buffer 1 multiplied
-            mbar_init(b0 + 48, 1);                   // second result ready
-        }
-        mbar_init(bar_drain, 1);
-        *abort_flag = 0;
-        fence_barrier_init();
-    }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(512) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    fence_proxy_async();          // the operand image was written with ordinary stores; the MMAs read it asynchronously
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // nothing starts before the weights are in place; if they never arrive every role skips its loop
+    const bool image_ok = mbar_wait(bar_img, 0u, abort_flag, a.st);
 
     ChainSlot slot[2];
 #pragma unroll
@@ -221,7 +226,7 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
         slot[s].nz = slot[s].np = slot[s].na = slot[s].nu = 0;
         slot[s].tile = -1;
     }
-    const int n_tiles = ceil_div(a.count, 128);
+    const int n_tiles = image_ok ? ceil_div(a.count, 128) : 0;
     // phases: W guide steps, then transition and emission hidden layer -- or gate, proposal (+ scale), first emission layer
     const int n_phases = LITERAL ? W + 3 : W + 2;
     const int ph_last = n_phases - 1;                             // its hidden layer goes to global memory, no second GEMM
