@@ -75,10 +75,12 @@ __device__ __forceinline__ uint32_t instr_desc_tf32(int n) {      // D = f32, A 
     return (1u << 4) | (2u << 7) | (2u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
+// Round to tf32 (nearest, ties away from zero) with two integer instructions instead of the conversion instruction,
+// which shares the slow special-function pipe with tanh: add half a unit of the 13 dropped bits to the magnitude,
+// clear them.  The same bits as cvt.rna.tf32.f32 for every finite value (an overflow of the mantissa carries into
+// the exponent, as it should).
 __device__ __forceinline__ float tf32_rna(float x) {
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);
 }
 
 __device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, float c, float d) {
