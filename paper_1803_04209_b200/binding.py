@@ -476,6 +476,23 @@ class Fitter:
             raise CutoffError(rc, "cutoff_elbo_grad")
         return self.elbo, self.grads
 
+    def capture_elbo_grad(self, xhat, eps):
+        """Capture elbo_grad(xhat, eps) in a CUDA graph.  xhat and eps are fixed tensors: the caller refills them (on the
+        current stream) before every replay_elbo_grad().  A step is some 150 small dependent launches, so a replay
+        costs a fraction of launching them one by one."""
+        import torch
+        self.elbo_grad(xhat, eps)                      # once outside the capture
+        torch.cuda.current_stream().synchronize()
+        self._graph_inputs = (xhat, eps)
+        self._graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self._graph):
+            self.elbo_grad(xhat, eps)
+
+    def replay_elbo_grad(self):
+        """Replay the captured step on the current contents of the captured input tensors; returns (elbo, grads)."""
+        self._graph.replay()
+        return self.elbo, self.grads
+
     def adam_step(self, lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, clip=10.0, grad_scale=None):
         """One Adam step on the negative mean ELBO (grad_scale = -1/batch) with clipping by the global norm."""
         import torch

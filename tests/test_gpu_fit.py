@@ -64,6 +64,32 @@ def test_elbo_and_gradient_match_the_oracle(N, D, H, lag, B):
     assert torch.equal(before, grads3)
 
 
+def test_graph_replay_of_the_step_equals_the_plain_call():
+    import torch
+    N, D, H, lag, B = 128, 8, 128, 2, 16
+    w, x, eps = _case(N, D, H, lag, B, seed=77)
+    plain = binding.Fitter(N, D, H, lag, B, w)
+    e_ref, g_ref = plain.elbo_grad(torch.from_numpy(x).cuda(), torch.from_numpy(eps).cuda())
+    torch.cuda.synchronize()
+    e_ref, g_ref = e_ref.clone(), g_ref.clone()
+    fitter = binding.Fitter(N, D, H, lag, B, w)
+    xs, es = torch.zeros((B, lag + 1, N), device="cuda"), torch.zeros((B, lag + 1, D), device="cuda")
+    fitter.capture_elbo_grad(xs, es)                      # captured on other contents
+    xs.copy_(torch.from_numpy(x)); es.copy_(torch.from_numpy(eps))
+    e1, g1 = fitter.replay_elbo_grad()
+    torch.cuda.synchronize()
+    assert torch.equal(e1, e_ref) and torch.equal(g1, g_ref)
+    # a second replay on new inputs follows them; back on the first inputs it gives the first result again
+    xs.mul_(1.01)
+    e2, _ = fitter.replay_elbo_grad()
+    torch.cuda.synchronize()
+    assert not torch.equal(e2, e_ref)
+    xs.copy_(torch.from_numpy(x))
+    e3, g3 = fitter.replay_elbo_grad()
+    torch.cuda.synchronize()
+    assert torch.equal(e3, e_ref) and torch.equal(g3, g_ref)
+
+
 def test_adam_steps_with_clipping_match_the_oracle():
     import torch
     N, D, H, lag, B = 24, 4, 16, 1, 12
