@@ -500,10 +500,11 @@ void launch_encoder(cutoff_ctx* c) {
         case 32: launch_rnn_resident<8>(c); break;
         case 64: launch_rnn_resident<16>(c); break;
         case 128: launch_rnn_resident<32>(c); break;
-        case 256: launch_rnn_resident<64>(c); break;
         default: {
+            // H = 256: a thread's 64 weights no longer fit its registers beside 1023 other threads; the cluster does
+            // the step in less time than one CTA that keeps half of the matrix in shared memory (17 against 21 us)
             const size_t cluster_smem = enc_rnn_cluster_smem_floats(c->H, c->W) * sizeof(float);
-            if (!fits && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024) {
+            if ((!fits || c->H == 256) && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024) {
                 // the matrix of a direction split over a cluster of 8 CTAs
                 k_enc_rnn_cluster<<<2 * kRnnClusterSize, c->H, cluster_smem, c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
             } else {
@@ -626,7 +627,6 @@ cudaError_t set_kernel_attributes(const cutoff_ctx* c) {
         case 32: e = allow_smem(k_enc_rnn_resident<8>, 200 * 1024); break;
         case 64: e = allow_smem(k_enc_rnn_resident<16>, 200 * 1024); break;
         case 128: e = allow_smem(k_enc_rnn_resident<32>, 200 * 1024); break;
-        case 256: e = allow_smem(k_enc_rnn_resident<64>, 200 * 1024); break;
         default: break;
     }
     if (e == cudaSuccess) e = allow_smem(k_enc_rnn_cluster, 200 * 1024);
@@ -867,7 +867,7 @@ int cutoff_load_weights(cutoff_ctx* c, const void* blob, size_t nbytes) {
     }
     CU_CHECK(c, cudaMemcpy(c->d_WT, wT.data(), wT.size() * sizeof(float), cudaMemcpyHostToDevice));
 
-    if (H == 32 || H == 64 || H == 128 || H == 256) {
+    if (H == 32 || H == 64 || H == 128) {
         // recurrence matrices regrouped per thread of k_enc_rnn_resident (the widths that kernel serves; the layout
         // needs H / 4 to be a multiple of 4): [dir][j4][thread = 4*i + q][4]
         const size_t HQ = H / 4, T = 4 * H;

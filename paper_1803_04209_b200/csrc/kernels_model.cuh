@@ -234,37 +234,32 @@ __global__ void __launch_bounds__(kRnnThreads) k_enc_rnn(ModelDev m, const float
 }
 
 // ---------------------------------------------------------------------------------------------
-// Encoder, part 2, latency version for H <= 256: the recurrence matrix never leaves the SM.
-// One CTA per direction, 4 threads per hidden unit; thread (i, q) owns columns q*H/4 .. of row i:
-// the first 32 of them in registers, the rest (H = 256 only) in shared memory, laid out
-// [column group][thread] so that a warp's 16-byte reads are contiguous.  The state is
-// double-buffered in shared memory, so a step costs one __syncthreads.
+// Encoder, part 2, latency version for H <= 128: the recurrence matrix never leaves the registers.
+// One CTA per direction, 4 threads per hidden unit; thread (i, q) owns columns q*H/4 .. of row i.
+// The state is double-buffered in shared memory, so a step costs one __syncthreads.
 // ---------------------------------------------------------------------------------------------
-template <int HQ>   // HQ = H / 4
+template <int HQ>   // HQ = H / 4 <= 32
 __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const float* __restrict__ wh_threads,
                                                               const float* __restrict__ proj,
                                                               const DevState* __restrict__ dev_state,
                                                               float* __restrict__ hlr /*[2][W][H]*/) {
-    constexpr int H = 4 * HQ, T = 16 * HQ, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ, PAD = HQ + 4;
+    static_assert(HQ <= 32, "a thread keeps its HQ weights in registers");
+    constexpr int H = 4 * HQ, T = 16 * HQ, PAD = HQ + 4;
     extern __shared__ __align__(16) float sm_rr[];
     float* state = sm_rr;                         // [2][4][PAD]
     float* sproj = state + 2 * 4 * PAD;           // [W][H]
-    float* swh = sproj + m.W * H;                 // [SQ/4][T][4]
     const int dir = blockIdx.x;
     const int t = threadIdx.x, i = t >> 2, q = t & 3;
     // wh_threads holds both recurrence matrices regrouped per thread, [dir][j4][thread][4]: the j4-th group of
     // four weights of thread (i, q) is Wh[i][q*HQ + 4*j4 ..], so that consecutive threads read consecutive 16 bytes
     const float4* Wh = reinterpret_cast<const float4*>(wh_threads) + static_cast<size_t>(dir) * (HQ / 4) * T;
     const float* init = dir ? m.b0 : m.a0;
-    float w[RQ];
+    float w[HQ];
 #pragma unroll
-    for (int j4 = 0; j4 < RQ / 4; ++j4) {
+    for (int j4 = 0; j4 < HQ / 4; ++j4) {
         const float4 v = Wh[static_cast<size_t>(j4) * T + t];
         w[4 * j4 + 0] = v.x; w[4 * j4 + 1] = v.y; w[4 * j4 + 2] = v.z; w[4 * j4 + 3] = v.w;
     }
-#pragma unroll
-    for (int j4 = 0; j4 < SQ / 4; ++j4)
-        *reinterpret_cast<float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4) = Wh[static_cast<size_t>(RQ / 4 + j4) * T + t];
     {
         const uint32_t pushes = dev_state->push_count;
         const float inv_scale = dev_state->inv_scale;
@@ -278,17 +273,10 @@ __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const 
         const float* st = state + cur * 4 * PAD + q * PAD;
         float acc = 0.0f;
 #pragma unroll
-        for (int j4 = 0; j4 < RQ / 4; ++j4) {
+        for (int j4 = 0; j4 < HQ / 4; ++j4) {
             const float4 v = *reinterpret_cast<const float4*>(st + 4 * j4);
             acc = fmaf(w[4 * j4 + 0], v.x, acc); acc = fmaf(w[4 * j4 + 1], v.y, acc);
             acc = fmaf(w[4 * j4 + 2], v.z, acc); acc = fmaf(w[4 * j4 + 3], v.w, acc);
-        }
-#pragma unroll
-        for (int j4 = 0; j4 < SQ / 4; ++j4) {
-            const float4 v = *reinterpret_cast<const float4*>(st + RQ + 4 * j4);
-            const float4 ww = *reinterpret_cast<const float4*>(swh + (static_cast<size_t>(j4) * T + t) * 4);
-            acc = fmaf(ww.x, v.x, acc); acc = fmaf(ww.y, v.y, acc);
-            acc = fmaf(ww.z, v.z, acc); acc = fmaf(ww.w, v.w, acc);
         }
         acc += __shfl_xor_sync(0xffffffffu, acc, 1);
         acc += __shfl_xor_sync(0xffffffffu, acc, 2);
@@ -303,12 +291,11 @@ __global__ void __launch_bounds__(16 * HQ) k_enc_rnn_resident(ModelDev m, const 
 }
 
 inline size_t enc_rnn_resident_smem_floats(int H, int W) {
-    const int HQ = H / 4, RQ = HQ < 32 ? HQ : 32, SQ = HQ - RQ;
-    return 2 * 4 * (HQ + 4) + static_cast<size_t>(W) * H + static_cast<size_t>(SQ) * 4 * H;
+    return 2 * 4 * (H / 4 + 4) + static_cast<size_t>(W) * H;
 }
 
 // ---------------------------------------------------------------------------------------------
-// Encoder, part 2, for 256 < H <= 640: the recurrence matrix of a direction is split over the shared
+// Encoder, part 2, for 256 <= H <= 640: the recurrence matrix of a direction is split over the shared
 // memories of a cluster of 8 CTAs (H/8 rows each), so it is read from global memory once.  Every CTA
 // keeps the whole state (double-buffered); after a step each row's new value is written into the next
 // state buffer of all 8 CTAs through distributed shared memory, and one cluster barrier (a hardware
