@@ -495,23 +495,18 @@ void refresh_projections(cutoff_ctx* c) {
 
 void launch_encoder(cutoff_ctx* c) {
     refresh_projections(c);
-    const bool fits = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float) <= 200 * 1024;
-    switch (fits ? c->H : 0) {
-        case 32: launch_rnn_resident<8>(c); break;
-        case 64: launch_rnn_resident<16>(c); break;
-        case 128: launch_rnn_resident<32>(c); break;
-        default: {
-            // H = 256: a thread's 64 weights no longer fit its registers beside 1023 other threads; the cluster does
-            // the step in less time than one CTA that keeps half of the matrix in shared memory (17 against 21 us)
-            const size_t cluster_smem = enc_rnn_cluster_smem_floats(c->H, c->W) * sizeof(float);
-            if ((!fits || c->H == 256) && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024) {
-                // the matrix of a direction split over a cluster of 8 CTAs
-                k_enc_rnn_cluster<<<2 * kRnnClusterSize, c->H, cluster_smem, c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
-            } else {
-                k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
-            }
-        }
-    }
+    // H <= 128: one CTA per direction with the recurrence matrix in registers.  From H = 256 on a thread's share no
+    // longer fits its registers, and a cluster of 8 CTAs per direction does the step in less time than one CTA that
+    // keeps part of the matrix in shared memory (H = 256: 17 against 21 us).
+    const size_t cluster_smem = enc_rnn_cluster_smem_floats(c->H, c->W) * sizeof(float);
+    const size_t resident_smem = enc_rnn_resident_smem_floats(c->H, c->W) * sizeof(float);
+    if (c->H == 32 && resident_smem <= 200 * 1024) launch_rnn_resident<8>(c);
+    else if (c->H == 64 && resident_smem <= 200 * 1024) launch_rnn_resident<16>(c);
+    else if (c->H == 128 && resident_smem <= 200 * 1024) launch_rnn_resident<32>(c);
+    else if (c->H >= 256 && c->H % 32 == 0 && c->H <= 1024 && cluster_smem <= 200 * 1024)
+        k_enc_rnn_cluster<<<2 * kRnnClusterSize, c->H, cluster_smem, c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
+    else
+        k_enc_rnn<<<2, kRnnThreads, 2 * c->H * sizeof(float), c->stream>>>(c->m, c->d_proj, c->d_state, c->d_hlr);
     c->launches += 1;
 }
 

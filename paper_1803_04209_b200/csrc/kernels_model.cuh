@@ -325,10 +325,19 @@ k_enc_rnn_cluster(ModelDev m, const float* __restrict__ proj, const DevState* __
     const int i = static_cast<int>(rank) * R + row;                    // hidden unit of this thread's row
     const float* Wh = (dir ? m.Whb : m.Whf) + static_cast<size_t>(rank) * R * H;
     const float* init = dir ? m.b0 : m.a0;
-    for (int idx = threadIdx.x; idx < R * (H / 4); idx += blockDim.x) {
-        const int r = idx / (H / 4), c = idx % (H / 4);
-        *reinterpret_cast<float4*>(sW + static_cast<size_t>(r) * ldw + 4 * c) =
-            *reinterpret_cast<const float4*>(Wh + static_cast<size_t>(r) * H + 4 * c);
+    // R * H / 4 = blockDim.x * H / 32 chunks of 16 bytes: every thread moves H / 32 of them, eight loads in flight
+    for (int base = 0; base < R * (H / 4); base += 8 * blockDim.x) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * blockDim.x + threadIdx.x;
+            if (idx < R * (H / 4)) v[u] = *reinterpret_cast<const float4*>(Wh + static_cast<size_t>(idx / (H / 4)) * H + 4 * (idx % (H / 4)));
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int idx = base + u * blockDim.x + threadIdx.x;
+            if (idx < R * (H / 4)) *reinterpret_cast<float4*>(sW + static_cast<size_t>(idx / (H / 4)) * ldw + 4 * (idx % (H / 4))) = v[u];
+        }
     }
     for (int k = threadIdx.x; k < H; k += blockDim.x) state[k] = init[k];
     {
@@ -344,13 +353,14 @@ k_enc_rnn_cluster(ModelDev m, const float* __restrict__ proj, const DevState* __
     for (int s = 0; s < W; ++s) {
         const int t = dir ? (W - 1 - s) : s;
         const float* st = state + cur * H;
-        float acc = 0.0f;
+        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;      // four chains: the sum's order is fixed all the same
         for (int c = part; c < H / 4; c += 8) {
             const float4 w = *reinterpret_cast<const float4*>(wrow + 4 * c);
             const float4 v = *reinterpret_cast<const float4*>(st + 4 * c);
-            acc = fmaf(w.x, v.x, acc); acc = fmaf(w.y, v.y, acc);
-            acc = fmaf(w.z, v.z, acc); acc = fmaf(w.w, v.w, acc);
+            a0 = fmaf(w.x, v.x, a0); a1 = fmaf(w.y, v.y, a1);
+            a2 = fmaf(w.z, v.z, a2); a3 = fmaf(w.w, v.w, a3);
         }
+        float acc = (a0 + a1) + (a2 + a3);
         acc += __shfl_xor_sync(0xffffffffu, acc, 1);
         acc += __shfl_xor_sync(0xffffffffu, acc, 2);
         acc += __shfl_xor_sync(0xffffffffu, acc, 4);
