@@ -516,6 +516,23 @@ def test_limits_of_the_supported_shapes(N, D, H, lag, S, prec):
     assert_decision_close(gpu, orc.predict(), N)
 
 
+@pytest.mark.parametrize("H,lag", [(256, 4), (288, 3), (320, 2), (384, 5), (512, 0), (576, 1), (640, 2)])
+def test_encoder_widths_on_the_cluster_kernel(H, lag):
+    # hidden widths from 256 up whose recurrence runs on the cluster of 8 CTAs per direction (rows split 8 ways,
+    # state exchanged through distributed shared memory), widths that are not powers of two included
+    N, D, S = 40, 8, 96
+    w = inputs.make_weights(N, D, H, seed=H, fan_in_ref=32)
+    trace = inputs.make_trace(N, lag + 4, seed=H + 1, sigma=0.2)
+    gpu = binding.Cutoff(N, D, H, lag, S, precision=0, seed=SEED)
+    gpu.load_weights(w)
+    orc = O.CutoffOracle(w, lag, S, seed=SEED)
+    for x in trace:
+        gpu.push(x)
+        orc.push(x)
+    assert_samples_close(gpu.debug_samples(0, S), orc.samples(np.arange(S)), TOL_X[0])
+    assert_decision_close(gpu, orc.predict(), N)
+
+
 @pytest.mark.parametrize("kw", [dict(n_workers=4097), dict(latent_dim=5), dict(latent_dim=64), dict(hidden=1028),
                                 dict(hidden=30), dict(lag=256), dict(latent_dim=32, hidden=1024)])
 def test_unsupported_shapes_are_refused(kw):
