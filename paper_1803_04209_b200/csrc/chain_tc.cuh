@@ -179,6 +179,15 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
             bulk_load_1d(base + off, reinterpret_cast<const uint8_t*>(a.image) + off, n, bar_img);
         }
     }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(512) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    // up to here nothing an earlier kernel of the stream writes has been touched (the image and the biases are
+    // weights): the encoder's states and the device state come after this point
+    dependency_wait();
+    launch_dependents();
     {
         for (int i = threadIdx.x; i < H; i += kChainTcThreads) {
             sbzs[i] = a.bz[i];
@@ -203,11 +212,6 @@ __global__ void __launch_bounds__(kChainTcThreads, 1) k_chain_tc(ChainTcArgs a) 
             }
         }
         if (!LITERAL && threadIdx.x < 32) sb2[threadIdx.x] = a.b2[threadIdx.x];
-    }
-    if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(512) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();

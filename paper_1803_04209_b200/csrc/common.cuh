@@ -19,6 +19,13 @@ struct DevState {
     uint32_t ticket;        // CTAs that have finished their column sums (self-resetting)
 };
 
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may begin while its
+// predecessor in the stream is still running, once every CTA of the predecessor has called launch_dependents (or
+// exited).  Whatever it does before dependency_wait() must not touch anything an earlier kernel writes; after it
+// the predecessor has completed and its writes are visible.  Both are no-ops in a kernel launched the plain way.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 constexpr int kErrBadValue = 1;
 constexpr int kErrTimeout = 2;
 constexpr int kErrNoFinisher = 4;   // a censored push in which every worker was censored

@@ -206,6 +206,23 @@ void put_second_layer(float* tiles, const float* w, size_t out_rows, size_t H, s
             for (size_t jj = 0; jj < 32; ++jj) tiles[kb * block_rows * 32 + swz(o, jj)] = host_tf32(w[o * H + kb * 32 + jj]);
 }
 
+// Launch `kernel` so that it may begin while the kernel before it in the stream is still running (programmatic
+// dependent launch): the kernel itself waits, by dependency_wait(), before it touches that kernel's results.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 int next_pow2(int n) {
     int p = 1;
     while (p < n) p <<= 1;
@@ -251,8 +268,8 @@ void plan_chunks(cutoff_ctx* c, int chunk_rows_wanted) {
 template <int E, bool SQ>
 void launch_sort_warp_sq(cutoff_ctx* c, int count, float* partial) {
     const size_t smem = sort_tma_smem_bytes<E>(c->ldx);
-    k_sort_sum_tma<E, SQ><<<c->sort_grid, kSortWarps * 32, smem, c->stream>>>(
-        c->d_x, c->ldx, c->N, count, partial, partial + static_cast<size_t>(kPartialRows) * c->N, c->d_state);
+    launch_dependent(k_sort_sum_tma<E, SQ>, dim3(c->sort_grid), dim3(kSortWarps * 32), smem, c->stream,
+                     c->d_x, c->ldx, c->N, count, partial, partial + static_cast<size_t>(kPartialRows) * c->N, c->d_state);
 }
 
 template <int E>
@@ -317,8 +334,8 @@ void launch_chain_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
     a.sample_base = sample_base; a.count = count; a.H = c->H; a.W = c->W; a.round_v = 1; a.v_out = c->d_v;
     const int tiles = ceil_div(count, 128);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    if (c->chain_tcl) tc::k_chain_tc<true><<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W, true), c->stream>>>(a);
-    else tc::k_chain_tc<false><<<grid, tc::kChainTcThreads, tc::chain_tc_smem_bytes(c->H, c->W), c->stream>>>(a);
+    if (c->chain_tcl) launch_dependent(tc::k_chain_tc<true>, dim3(grid), dim3(tc::kChainTcThreads), tc::chain_tc_smem_bytes(c->H, c->W, true), c->stream, a);
+    else launch_dependent(tc::k_chain_tc<false>, dim3(grid), dim3(tc::kChainTcThreads), tc::chain_tc_smem_bytes(c->H, c->W), c->stream, a);
     c->launches += 1;
 }
 
@@ -421,7 +438,7 @@ void launch_emission_tc(cutoff_ctx* c, uint32_t sample_base, int count) {
     }
     const int tiles = ceil_div(c->N, tc::kBW) * ceil_div(count, tc::kBM);
     const int grid = tiles < c->sm_count ? tiles : c->sm_count;
-    tc::k_emit_tc<<<grid, tc::kThreads, tc::kSmemBytes, c->stream>>>(c->map_v, c->map_w4, a);
+    launch_dependent(tc::k_emit_tc, dim3(grid), dim3(tc::kThreads), tc::kSmemBytes, c->stream, c->map_v, c->map_w4, a);
     c->launches += 1;
 }
 
@@ -543,11 +560,10 @@ int enqueue_decision(cutoff_ctx* c, bool decide = true) {
         if (timed) cudaEventRecord(c->ev[4][ch], c->stream);
     }
     const int64_t total = c->cfg.total_samples > 0 ? c->cfg.total_samples : c->S;
-    k_colsum_decide<<<ceil_div(c->N, 32), kColsumThreads, 0, c->stream>>>(c->d_partial, c->n_chunks * c->sort_grid, c->N,
-                                                                         c->d_sums, 1.0 / static_cast<double>(total),
-                                                                         c->d_state, c->d_E, c->d_omega,
-                                                                         c->want_std ? c->d_partial + static_cast<size_t>(kPartialRows) * c->N : nullptr,
-                                                                         c->d_std, decide ? 1 : 0);
+    launch_dependent(k_colsum_decide, dim3(ceil_div(c->N, 32)), dim3(kColsumThreads), 0, c->stream,
+                     c->d_partial, c->n_chunks * c->sort_grid, c->N, c->d_sums, 1.0 / static_cast<double>(total), c->d_state,
+                     c->d_E, c->d_omega, c->want_std ? c->d_partial + static_cast<size_t>(kPartialRows) * c->N : nullptr,
+                     c->d_std, decide ? 1 : 0);
     c->have_std = c->want_std;
     c->launches += 1;
     if (timed) cudaEventRecord(c->ev[5][0], c->stream);

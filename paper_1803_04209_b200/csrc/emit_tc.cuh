@@ -222,6 +222,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_emit_tc(const __grid_constant__
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    dependency_wait();            // the hidden vectors and the device state are an earlier kernel's
+    launch_dependents();
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------------------------------------------------

@@ -314,6 +314,7 @@ __global__ void __cluster_dims__(kRnnClusterSize, 1, 1) __launch_bounds__(1024)
 k_enc_rnn_cluster(ModelDev m, const float* __restrict__ proj, const DevState* __restrict__ dev_state,
                   float* __restrict__ hlr /*[2][W][H]*/) {
     extern __shared__ __align__(16) float sm_rc[];
+    launch_dependents();      // the chain kernel may set itself up on the SMs this kernel leaves free
     const int H = m.H, W = m.W, R = H / kRnnClusterSize, ldw = H + 8;
     float* sW = sm_rc;                         // [R][ldw]  rows rank*R .. of the recurrence matrix
     float* state = sW + static_cast<size_t>(R) * ldw;      // [2][H]

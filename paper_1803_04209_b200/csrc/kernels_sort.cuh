@@ -307,6 +307,8 @@ __global__ void __launch_bounds__(kSortWarps * 32) k_sort_sum_tma(const float* _
         fence_proxy_async();
     }
     __syncthreads();
+    dependency_wait();            // the sample matrix is an earlier kernel's
+    launch_dependents();
 
     float acc[E], acc_sq[SQ ? E : 1];
 #pragma unroll
@@ -494,6 +496,7 @@ __global__ void __launch_bounds__(kColsumThreads) k_colsum_decide(const float* _
                                                                    float* __restrict__ std_out, int decide) {
     __shared__ double red[kColsumSlices][32];
     __shared__ bool is_last;
+    dependency_wait();            // the partial rows are an earlier kernel's
     const int col = blockIdx.x * 32 + (threadIdx.x & 31), slice = threadIdx.x >> 5;
     if (partial_sq) {
         // spread of each order statistic over the samples: sqrt(E[x^2] - E[x]^2), in seconds
