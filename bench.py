@@ -37,7 +37,7 @@ MINMAX_LANES_PER_SM = 64         # fp32 min / max lanes per SM per clock (ALU pi
 # kernel as committed with that summary; set to None when the kernel changes): the sample matrix read once
 # (grows with S) plus the partial rows written (one per CTA: does not grow with S).
 NCU_TRAFFIC = {
-    ("n1024", "sort"): {"bytes_per_sample": 201393664 / 49152, "bytes_fixed": 3926784,
+    ("n1024", "sort"): {"bytes_per_sample": 201400064 / 49152, "bytes_fixed": 4353792,
                         "source": "profiles/ncu_full_n1024_s49152_chain_emit_sort.txt (S=49152, scaled by S)"},
     ("n4096", "sort"): {"bytes_per_sample": 134251776 / 8192, "bytes_fixed": 8298752,
                         "source": "profiles/ncu_full_n4096_s8192_sort.txt (S=8192, scaled by S)"},
